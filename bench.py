@@ -35,8 +35,8 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-# DRAM bytes per algorithmic byte of st_k_decode, from the ncu capture summarised in profiles/st_k_decode_small_case.md
-# (272.8 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
+# DRAM bytes per algorithmic byte of st_k_decode, from an ncu capture of the small decode case (--profile-case decode:
+# 272.8 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.0177
 
 METRIC = "reasoning-decode tok/s per layer (chunk prefill concurrent on a second stream)"
@@ -469,8 +469,8 @@ def main():
     roofline = {"bound": "hbm", "kernel": "st_k_decode", "achieved": dec_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": dec_gbs / peaks["hbm_gbs"], "of": peaks["source"],
                 "traffic": DECODE_DRAM_PER_ALGORITHMIC_BYTE * dec_bytes_per_launch,
-                "traffic_how": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the small case in "
-                               "profiles/st_k_decode_small_case.md, scaled by the K/V bytes one launch streams",
+                "traffic_how": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the small decode case "
+                               "(--profile-case decode), scaled by the K/V bytes one launch streams",
                 "launches": dec_launches * L * args.steps, "launches_timed": n_dec, "avg_launch_us": dec_avg_s * 1e6,
                 "algorithmic_bytes_per_launch": dec_bytes_per_launch,
                 "timed": "every %d-th launch, its own bytes over its own time" % period,

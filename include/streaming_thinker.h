@@ -19,7 +19,10 @@
  *     [tokens][heads][128]; out is fp32 [tokens][n_q_heads][128]. The caller owns them.
  *   - Calls are asynchronous on the cudaStream_t passed as `stream` (NULL = legacy default
  *     stream). Every argument is validated on the host before anything is launched; a call
- *     that fails changes no state.
+ *     that fails changes no state. That holds for a CUDA runtime failure in the middle of a call
+ *     (ST_ERR_CUDA) too: pages the call had taken return to the free list and its step is no longer
+ *     pending, so the same call can be issued again; work it had already queued on the stream is not
+ *     recalled (it only rewrites page-table entries and cache slots that the repeated call writes again).
  *   - One context is driven from one host thread. All source-side calls
  *     (st_append_source_chunk) must be stream-ordered among themselves, and so must all
  *     reasoning-side calls (st_reason_decode, st_reason_extend); the two sides may use two
@@ -51,9 +54,17 @@ extern "C" {
 #define ST_ERR_STATE          -4   /* layer out of order, or step arguments differ between layers        */
 #define ST_ERR_CUDA           -5   /* a CUDA runtime call failed                                          */
 #define ST_ERR_DEVICE_TIMEOUT -6   /* a bounded device-side wait expired (reported by st_device_status)  */
+#define ST_ERR_DEVICE_CHECK   -7   /* a device-side bounds check failed: a page id read from a page table
+                                      lies outside its pool. The access was skipped, nothing faulted; rows
+                                      of the call are undefined (reported by st_device_status)            */
 
 /* st_config.flags */
 #define ST_CFG_HOST_ONLY       1u  /* plan only: no device memory, no launches (host logic and its tests) */
+#define ST_CFG_DEBUG_CHECKS    2u  /* debug context: free pages (at st_create, and again when st_reset releases
+                                      them) hold a large finite sentinel (bf16 9.95e29) instead of zeros, so
+                                      that a key or value read from beyond the visible ranges -- which the
+                                      kernels would otherwise multiply by a weight of zero without a trace --
+                                      shows up in the rows. The kernels' page-id checks are always on.     */
 /* per-call flags */
 #define ST_END_OF_UNIT         1u  /* source side: this chunk completes a source unit (N_EOS += 1);
                                       reasoning side: the unit's boundary token was produced (N_EOT += 1) */
@@ -195,9 +206,23 @@ ST_API int st_debug_page_table(const st_ctx *ctx, int32_t seq_id, int32_t which,
  * ST_ERR_DEVICE_TIMEOUT once and the context is usable as before. Nothing faults, traps or spins without bound. */
 ST_API int st_debug_wait_expiry(st_ctx *ctx, int32_t limit_ms, void *stream);
 
-/* Device-side status word: ST_OK, or ST_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait since the
- * last call of this function (which clears it). Synchronises the device. */
+/* Device-side status word: ST_OK, ST_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait, or
+ * ST_ERR_DEVICE_CHECK if a kernel met a page id outside its pool, since the last call of this function
+ * (which clears it). Synchronises the device. */
 ST_API int st_device_status(st_ctx *ctx);
+
+/* Test surface for the failure path of the attention calls: the n_steps-th device step issued from now on
+ * (stream wait, page-table update, staging copy, append launch, attention launch; counted across calls)
+ * fails on the host with ST_ERR_CUDA before it does anything, as a failing CUDA runtime call would.
+ * n_steps = 0 disarms. Works on host-only contexts too. */
+ST_API int st_debug_fail_after(st_ctx *ctx, int32_t n_steps);
+
+/* Test surface for the kernels' page-id check: overwrites entry `index` of the device page table of
+ * sequence seq_id (which = 0 source, 1 reasoning) with `page`, which may lie outside the pool. The next
+ * kernel that reads the entry records ST_ERR_DEVICE_CHECK and skips the access. The host-side table is
+ * not changed; st_reset followed by new appends rewrites the entry. Synchronises `stream`. */
+ST_API int st_debug_corrupt_page_table(st_ctx *ctx, int32_t seq_id, int32_t which, int32_t index, int32_t page,
+                                       void *stream);
 
 /* Kernel timing for benchmarks. While enabled (every > 0), launches of the two dominant kernels are
  * bracketed by CUDA events on the stream they are launched on: every `every`-th launch of the dual-cache
@@ -232,28 +257,46 @@ ST_API const char *st_last_error_string(const st_ctx *ctx);
  * which must already be in the reasoning cache), exactly the row st_reason_decode produces.
  *
  * Inputs (device unless stated): pool_source / pool_reason = first byte of the layer's page blocks in each
- * pool (block of page p, kv head h at ((p * n_kv_heads) + h) * 32768; see "Pool layout" below);
- * page_table_* = int32 [slot][table_stride_*] page ids; slots / source_len / reason_len = HOST arrays of
- * n_seq ints (page-table row, visible source tokens, reasoning tokens); q_rotated = bf16
- * [n_seq][n_q_heads][128], already rotated at position reason_len[b] - 1; out = fp32 [n_seq][n_q_heads][128].
- * softmax_scale 0 means 1/sqrt(128). err / err_cap: optional HOST buffer that receives a message on failure.
+ * pool (block of page p, kv head h at ((p * n_kv_heads) + h) * 32768; see "Pool layout" below), holding
+ * n_pages_source / n_pages_reason pages; page_table_* = int32 [slot][table_stride_*] page ids;
+ * slots / source_len / reason_len = HOST arrays of n_seq ints (page-table row, visible source tokens,
+ * reasoning tokens); q_rotated = bf16 [n_seq][n_q_heads][128], already rotated at position
+ * reason_len[b] - 1; out = fp32 [n_seq][n_q_heads][128]. softmax_scale 0 means 1/sqrt(128).
+ * err / err_cap: optional HOST buffer that receives a message on failure.
+ *
+ * The page tables are the caller's, so the kernel checks every page id it reads against n_pages_* before it
+ * builds an address from it: an id outside the pool is never dereferenced; the kernel stops, and
+ * st_decode_static_status reports ST_ERR_DEVICE_CHECK (rows of that call are undefined, rows that only the
+ * merge kernel would have written stay untouched). The same word reports a bounded wait that ran out
+ * (ST_ERR_DEVICE_TIMEOUT). The call itself returns before the kernels have run and cannot report either.
  *
  * Limits: n_seq <= 112 and n_seq * n_kv_heads <= 512 per call; larger calls are rejected with
  * ST_ERR_INVALID_ARG and a message. The first call on a device looks up the address of the built-in array and
  * sets kernel attributes for that device, so make that first call outside any stream capture. All calls on a
  * GPU share the one array, which keeps the previous call's contents (the call clears the only word that must
  * start at zero): calls that overlap in time on the same GPU -- from different streams or threads -- race and
- * give wrong results; order them on one stream or with events.
+ * give wrong results; order them on one stream or with events. The call makes `device` current while it
+ * runs and restores the caller's current device before it returns.
  *
  * Pool layout (also what cfg->pool_base holds): the source pool, then the reasoning pool; each pool is
  * [layer][page][kv head] blocks of 32768 bytes. */
-ST_API int st_decode_attention_static(int32_t device, const void *pool_source, const void *pool_reason,
+ST_API int st_decode_attention_static(int32_t device, const void *pool_source, int64_t n_pages_source,
+                                      const void *pool_reason, int64_t n_pages_reason,
                                       const int32_t *page_table_source, int32_t table_stride_source,
                                       const int32_t *page_table_reason, int32_t table_stride_reason,
                                       const int32_t *slots, const int32_t *source_len, const int32_t *reason_len,
                                       int32_t n_seq, const void *q_rotated, void *out, int32_t n_q_heads,
                                       int32_t n_kv_heads, float softmax_scale, void *stream, char *err,
                                       int32_t err_cap);
+
+/* Status of the most recent st_decode_attention_static call on `device` (every such call clears the word when
+ * its work starts on the stream, so read it before queueing the next call if each call is to be checked):
+ * waits for `stream` (the stream the call was queued on) and reads the status word of the built-in workspace.
+ * Returns ST_OK,
+ * ST_ERR_DEVICE_CHECK (a page id outside its pool was met; the access was skipped), ST_ERR_DEVICE_TIMEOUT (a
+ * bounded wait inside the kernels ran out), ST_ERR_INVALID_ARG (no such call has been made on the device) or
+ * ST_ERR_CUDA. Like the call it reports on, it allocates nothing; the paper has no counterpart. */
+ST_API int st_decode_static_status(int32_t device, void *stream);
 
 #ifdef __cplusplus
 }

@@ -224,12 +224,6 @@ def attention_rows(sched: Schedule, q, k, v, rows, theta: float = 1.0e6, scale=N
     return (O, probs) if return_probs else O
 
 
-def attention_all(sched: Schedule, q, k, v, **kw):
-    """Every row; returns ``(O_source[S,Hq,d], O_reasoning[R,Hq,d])``."""
-    O = attention_rows(sched, q, k, v, np.arange(sched.S + sched.R), **kw)
-    return O[: sched.S], O[sched.S :]
-
-
 def expected_cache(sched: Schedule, k, v, theta: float = 1.0e6):
     """What the two caches must hold: ``bf16(RoPE(k, pos))`` and ``v``, split by stream."""
     kh = round_to_bf16(rope(k, sched.pos_ids, theta))

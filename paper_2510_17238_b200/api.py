@@ -19,13 +19,13 @@ if not os.path.exists(_LIB_PATH):
 lib = C.CDLL(_LIB_PATH)
 
 ST_OK, ST_ERR_INVALID_ARG, ST_ERR_OOM_PAGES, ST_ERR_NOT_READY = 0, -1, -2, -3
-ST_ERR_STATE, ST_ERR_CUDA, ST_ERR_DEVICE_TIMEOUT = -4, -5, -6
-ST_CFG_HOST_ONLY = 1
+ST_ERR_STATE, ST_ERR_CUDA, ST_ERR_DEVICE_TIMEOUT, ST_ERR_DEVICE_CHECK = -4, -5, -6, -7
+ST_CFG_HOST_ONLY, ST_CFG_DEBUG_CHECKS = 1, 2
 ST_END_OF_UNIT, ST_REFERENCE_KERNELS, ST_IO_HOST = 1, 2, 4
 ST_VIS_DEFAULT, ST_VIS_ALL = -1, -2
 
 ERROR_NAMES = {0: "ST_OK", -1: "ST_ERR_INVALID_ARG", -2: "ST_ERR_OOM_PAGES", -3: "ST_ERR_NOT_READY",
-               -4: "ST_ERR_STATE", -5: "ST_ERR_CUDA", -6: "ST_ERR_DEVICE_TIMEOUT"}
+               -4: "ST_ERR_STATE", -5: "ST_ERR_CUDA", -6: "ST_ERR_DEVICE_TIMEOUT", -7: "ST_ERR_DEVICE_CHECK"}
 
 
 class st_config(C.Structure):
@@ -65,9 +65,12 @@ _SIGS = {
     "st_kernel_timing_read": (C.c_int, [_vp, C.c_int32, _i64p, C.POINTER(C.c_double)]),
     "st_launch_count": (C.c_int64, [_vp]),
     "st_last_error_string": (C.c_char_p, [_vp]),
-    "st_decode_attention_static": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_int32, _vp, C.c_int32, _i32p, _i32p, _i32p,
-                                             C.c_int32, _vp, _vp, C.c_int32, C.c_int32, C.c_float, _vp, C.c_char_p,
-                                             C.c_int32]),
+    "st_debug_fail_after": (C.c_int, [_vp, C.c_int32]),
+    "st_debug_corrupt_page_table": (C.c_int, [_vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp]),
+    "st_decode_attention_static": (C.c_int, [C.c_int32, _vp, C.c_int64, _vp, C.c_int64, _vp, C.c_int32, _vp, C.c_int32,
+                                             _i32p, _i32p, _i32p, C.c_int32, _vp, _vp, C.c_int32, C.c_int32, C.c_float,
+                                             _vp, C.c_char_p, C.c_int32]),
+    "st_decode_static_status": (C.c_int, [C.c_int32, _vp]),
 }
 EXPORTED = tuple(_SIGS)
 for _name, (_res, _args) in _SIGS.items():
@@ -209,6 +212,12 @@ class Context:
         rc = lib.st_debug_wait_expiry(self._h, int(limit_ms), _ptr(stream))
         return self._check(rc) if check else rc
 
+    def debug_fail_after(self, n_steps):
+        return self._check(lib.st_debug_fail_after(self._h, int(n_steps)))
+
+    def debug_corrupt_page_table(self, seq_id, which, index, page, stream=None):
+        return self._check(lib.st_debug_corrupt_page_table(self._h, seq_id, which, index, page, _ptr(stream)))
+
     def kernel_timing_enable(self, every=1):
         """Bracket every `every`-th launch of the two dominant kernels with CUDA events (0 / False = off)."""
         return self._check(lib.st_kernel_timing_enable(self._h, int(every)))
@@ -261,9 +270,9 @@ def schedule_dense_mask(src_unit_len, rsn_unit_len, final_len=0, lag_units=0):
     return mask[:T, :T]
 
 
-def decode_attention_static(device, pool_source, pool_reason, page_table_source, table_stride_source,
-                            page_table_reason, table_stride_reason, slots, source_len, reason_len, q_rotated, out,
-                            n_q_heads, n_kv_heads, softmax_scale=0.0, stream=None, check=True):
+def decode_attention_static(device, pool_source, n_pages_source, pool_reason, n_pages_reason, page_table_source,
+                            table_stride_source, page_table_reason, table_stride_reason, slots, source_len, reason_len,
+                            q_rotated, out, n_q_heads, n_kv_heads, softmax_scale=0.0, stream=None, check=True):
     """st_decode_attention_static: decode attention on the workspace built into the library (no allocation).
 
     Pointers may be torch tensors, numpy arrays or raw addresses; slots / source_len / reason_len are host
@@ -272,10 +281,15 @@ def decode_attention_static(device, pool_source, pool_reason, page_table_source,
     pa, ka = _i32(source_len)
     pr, kr = _i32(reason_len)
     err = C.create_string_buffer(256)
-    rc = lib.st_decode_attention_static(device, _ptr(pool_source), _ptr(pool_reason), _ptr(page_table_source),
-                                        table_stride_source, _ptr(page_table_reason), table_stride_reason, ps, pa, pr,
-                                        len(ks), _ptr(q_rotated), _ptr(out), n_q_heads, n_kv_heads, softmax_scale,
-                                        _ptr(stream), err, 256)
+    rc = lib.st_decode_attention_static(device, _ptr(pool_source), n_pages_source, _ptr(pool_reason), n_pages_reason,
+                                        _ptr(page_table_source), table_stride_source, _ptr(page_table_reason),
+                                        table_stride_reason, ps, pa, pr, len(ks), _ptr(q_rotated), _ptr(out), n_q_heads,
+                                        n_kv_heads, softmax_scale, _ptr(stream), err, 256)
     if rc != ST_OK and check:
         raise StError(rc, err.value.decode())
     return rc, err.value.decode()
+
+
+def decode_static_status(device, stream=None) -> int:
+    """st_decode_static_status: status code of the most recent allocation-free decode call on the device."""
+    return int(lib.st_decode_static_status(device, _ptr(stream)))

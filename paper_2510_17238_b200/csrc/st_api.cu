@@ -87,6 +87,8 @@ struct st_ctx {
   std::vector<int32_t> meta_pos, meta_vis_src, meta_vis_rsn;
   std::string err;
   int64_t launches = 0;
+  bool poison = false;           // ST_CFG_DEBUG_CHECKS: free pages hold a large finite sentinel instead of zeros
+  int fail_countdown = 0;        // test hook: the n-th internal device step from now reports ST_ERR_CUDA
 };
 
 namespace {
@@ -100,6 +102,14 @@ int fail(st_ctx *ctx, int code, const std::string &msg) {
     cudaError_t e__ = (call);                                                                 \
     if (e__ != cudaSuccess) return fail(ctx, ST_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__)); \
   } while (0)
+
+// Test hook (st_debug_fail_after): counts the device steps of a call (stream wait, page-table update, staging copy,
+// append launch, attention launch) and makes the chosen one fail on the host, as a CUDA error would.
+int injected_failure(st_ctx *ctx, const char *step) {
+  if (ctx->fail_countdown > 0 && --ctx->fail_countdown == 0)
+    return fail(ctx, ST_ERR_CUDA, std::string(step) + ": failure injected by st_debug_fail_after");
+  return ST_OK;
+}
 
 bool config_ok(const st_config *c, std::string *why) {
   auto bad = [&](const char *m) { if (why) *why = m; return false; };
@@ -215,7 +225,18 @@ int plan_pages(st_ctx *ctx, int which, const int32_t *seq_ids, const int32_t *cu
   return ST_OK;
 }
 
+// Undo plan_pages: the pages listed in `updates` (in allocation order) go back to the free list, newest first,
+// so that the free list is exactly what it was.
+void unplan_pages(st_ctx *ctx, const std::vector<st::PageUpdate> &updates) {
+  for (auto it = updates.rbegin(); it != updates.rend(); ++it) {
+    const int which = it->slot_which & 1, slot = it->slot_which >> 1;
+    ctx->seqs[slot].pages[which].pop_back();
+    ctx->free_pages[which].push_back(it->page);
+  }
+}
+
 int push_page_updates(st_ctx *ctx, const std::vector<st::PageUpdate> &updates, cudaStream_t stream) {
+  if (int rc = injected_failure(ctx, "page-table update")) return rc;
   if (ctx->host_only) return ST_OK;
   for (size_t off = 0; off < updates.size(); off += st::kMaxPageUpdates) {
     st::PageUpdateParams pp;
@@ -259,6 +280,7 @@ int resolve_visibility(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq, const
 
 // Make `stream` wait for the source append with the given serial if it ran on another stream.
 int wait_for_append(st_ctx *ctx, uint64_t serial, cudaStream_t stream) {
+  if (int rc = injected_failure(ctx, "stream wait")) return rc;
   if (ctx->host_only || serial == 0) return ST_OK;
   EventRec &rec = ctx->events[serial % kEventRing];
   if (rec.serial != serial) {
@@ -306,6 +328,7 @@ int stage_inputs(st_ctx *ctx, int side, uint32_t flags, int32_t total, const voi
   io->k = (const __nv_bfloat16 *)k;
   io->v = (const __nv_bfloat16 *)v;
   io->out = (float *)out;
+  if (int rc = injected_failure(ctx, "staging copy")) return rc;
   if (!(flags & ST_IO_HOST) || ctx->host_only || total == 0) return ST_OK;
   const size_t qb = (size_t)total * ctx->cfg.n_q_heads * 256, kb = (size_t)total * ctx->cfg.n_kv_heads * 256;
   if (qb + 2 * kb <= kInPlaceHostIoBytes) {
@@ -319,6 +342,14 @@ int stage_inputs(st_ctx *ctx, int side, uint32_t flags, int32_t total, const voi
       io->in_place = true;
       return ST_OK;
     }
+  }
+  if (!ctx->stage_q[side]) {
+    // staging buffers exist only for contexts that really stage host calls: allocated on the first such call of a side
+    const size_t T = ctx->cfg.max_tokens_per_call;
+    ST_CUDA(ctx, cudaMalloc(&ctx->stage_q[side], T * ctx->cfg.n_q_heads * 256));
+    ST_CUDA(ctx, cudaMalloc(&ctx->stage_k[side], T * ctx->cfg.n_kv_heads * 256));
+    ST_CUDA(ctx, cudaMalloc(&ctx->stage_v[side], T * ctx->cfg.n_kv_heads * 256));
+    ST_CUDA(ctx, cudaMalloc(&ctx->stage_out[side], T * ctx->cfg.n_q_heads * 512));
   }
   ST_CUDA(ctx, cudaMemcpyAsync(ctx->stage_q[side], q, qb, cudaMemcpyHostToDevice, stream));
   ST_CUDA(ctx, cudaMemcpyAsync(ctx->stage_k[side], k, kb, cudaMemcpyHostToDevice, stream));
@@ -339,6 +370,7 @@ int unstage_output(st_ctx *ctx, int side, uint32_t flags, int32_t total, void *o
 // Launch the append kernel (K and V into the cache of side `which`, rotated q into scratch).
 int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
                const IoPtrs &io, bool want_q, cudaStream_t stream) {
+  if (int rc = injected_failure(ctx, "append launch")) return rc;
   if (ctx->host_only) return ST_OK;
   for (int s0 = 0; s0 < n_seq; s0 += st::kMaxSeqPerLaunch) {
     const int ns = std::min<int>(st::kMaxSeqPerLaunch, n_seq - s0);
@@ -350,6 +382,8 @@ int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, co
     ap.pool = ctx->pool[which] + (size_t)layer * ctx->layer_stride[which];
     ap.ptab = ctx->d_ptab[which];
     ap.ptab_stride = ctx->ptab_stride[which];
+    ap.n_pages = (int32_t)(which ? ctx->cfg.n_pages_reason : ctx->cfg.n_pages_source);
+    ap.status = ctx->d_status;
     ap.n_seq = ns;
     ap.n_q_heads = ctx->cfg.n_q_heads;
     ap.n_kv_heads = ctx->cfg.n_kv_heads;
@@ -378,6 +412,8 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
   p->pool_b = ctx->pool[b] + (size_t)layer * ctx->layer_stride[b];
   p->ptab_b = ctx->d_ptab[b];
   p->ptab_stride_b = ctx->ptab_stride[b];
+  p->n_pages_a = (int32_t)ctx->cfg.n_pages_source;
+  p->n_pages_b = (int32_t)(b ? ctx->cfg.n_pages_reason : ctx->cfg.n_pages_source);
   p->qhat = ctx->qhat[side];
   p->q_raw = p->k_raw = p->v_raw = nullptr;
   p->rope_hi = p->rope_lo = nullptr;
@@ -396,6 +432,7 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
 int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
                   const std::vector<int32_t> &vis_tokens, float *out, uint32_t flags, cudaStream_t stream,
                   const IoPtrs *fused) {
+  if (int rc = injected_failure(ctx, "attention launch")) return rc;
   if (ctx->host_only || !out) return ST_OK;
   const int side = kind == 0 ? 0 : 1;
   const int total_rows = cu[n_seq];
@@ -511,32 +548,44 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     record_meta(ctx, kind, seq_ids, cu, n_seq, pd.vis_tokens);
   }
 
-  if (!ctx->host_only) ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
-  if (kind != 0 && (rc = wait_for_append(ctx, pd.wait_serial, stream))) return rc;
-  if ((rc = push_page_updates(ctx, updates, stream))) return rc;
-  IoPtrs io;
-  if ((rc = stage_inputs(ctx, side, flags, total, q, k, v, out, stream, &io))) return rc;
-  // A decode step's append (one token per sequence) runs inside the decode kernel: the step is then two kernels
-  // instead of three. Cache-only calls and the cross-check kernels keep the separate append.
-  const bool fuse_append = kind == 1 && io.out != nullptr && !(flags & ST_REFERENCE_KERNELS) && !ctx->host_only;
-  if (!fuse_append && (rc = run_append(ctx, side, layer, seq_ids, cu, n_seq, io, io.out != nullptr, stream))) return rc;
-  if ((rc = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, io.out, flags, stream,
-                          fuse_append ? &io : nullptr))) return rc;
-  if ((rc = unstage_output(ctx, side, flags, total, out, stream, io))) return rc;
+  // Device steps. If one of them fails, the host-side plan of this call is taken back (pages to the free list, the
+  // step no longer pending), so that the context is what it was before the call; work already queued stays queued.
+  uint64_t serial = 0;
+  auto device_steps = [&]() -> int {
+    int r;
+    if (!ctx->host_only) ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (kind != 0 && (r = wait_for_append(ctx, pd.wait_serial, stream))) return r;
+    if ((r = push_page_updates(ctx, updates, stream))) return r;
+    IoPtrs io;
+    if ((r = stage_inputs(ctx, side, flags, total, q, k, v, out, stream, &io))) return r;
+    // A decode step's append (one token per sequence) runs inside the decode kernel: the step is then two kernels
+    // instead of three. Cache-only calls and the cross-check kernels keep the separate append.
+    const bool fuse_append = kind == 1 && io.out != nullptr && !(flags & ST_REFERENCE_KERNELS) && !ctx->host_only;
+    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, io, io.out != nullptr, stream))) return r;
+    if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, io.out, flags, stream,
+                           fuse_append ? &io : nullptr))) return r;
+    if ((r = unstage_output(ctx, side, flags, total, out, stream, io))) return r;
+    if (layer == ctx->cfg.n_layers - 1 && kind == 0 && !ctx->host_only) {
+      // the event later reasoning-side calls wait for
+      EventRec &rec = ctx->events[(ctx->serial + 1) % kEventRing];
+      if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
+      ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
+      rec.stream = stream;
+      rec.serial = ctx->serial + 1;
+    }
+    return ST_OK;
+  };
+  if ((rc = device_steps())) {
+    if (layer == 0) {
+      unplan_pages(ctx, updates);
+      pd.active = false;
+    }
+    return rc;
+  }
 
   if (layer == ctx->cfg.n_layers - 1) {
     // commit the step
-    uint64_t serial = 0;
-    if (kind == 0) {
-      serial = ++ctx->serial;
-      if (!ctx->host_only) {
-        EventRec &rec = ctx->events[serial % kEventRing];
-        if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
-        ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
-        rec.stream = stream;
-        rec.serial = serial;
-      }
-    }
+    if (kind == 0) serial = ++ctx->serial;
     for (int b = 0; b < n_seq; ++b) {
       SeqState &sq = ctx->seqs[seq_ids[b]];
       sq.len[side] += cu[b + 1] - cu[b];
@@ -588,7 +637,7 @@ int st_create(const st_config *cfg, st_ctx **out) {
   if (!out) { g_create_error = "out is NULL"; return ST_ERR_INVALID_ARG; }
   *out = nullptr;
   if (!config_ok(cfg, &why)) { g_create_error = why; return ST_ERR_INVALID_ARG; }
-  if (cfg->flags & ~ST_CFG_HOST_ONLY) { g_create_error = "unknown config flag"; return ST_ERR_INVALID_ARG; }
+  if (cfg->flags & ~(ST_CFG_HOST_ONLY | ST_CFG_DEBUG_CHECKS)) { g_create_error = "unknown config flag"; return ST_ERR_INVALID_ARG; }
   const uint64_t pool_bytes = st_pool_bytes(cfg);
   if (cfg->pool_base && (cfg->pool_bytes < pool_bytes || ((uintptr_t)cfg->pool_base & 1023))) {
     g_create_error = "pool_base must be 1024-byte aligned and hold st_pool_bytes() bytes";
@@ -597,6 +646,7 @@ int st_create(const st_config *cfg, st_ctx **out) {
   st_ctx *ctx = new st_ctx();
   ctx->cfg = *cfg;
   ctx->host_only = (cfg->flags & ST_CFG_HOST_ONLY) != 0;
+  ctx->poison = (cfg->flags & ST_CFG_DEBUG_CHECKS) != 0;
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / sqrt((double)cfg->head_dim);
   ctx->scale_log2 = (float)(scale * 1.4426950408889634);
@@ -643,17 +693,19 @@ int st_create(const st_config *cfg, st_ctx **out) {
     }
     ctx->pool[0] = ctx->pool_alloc;
     ctx->pool[1] = ctx->pool_alloc + (size_t)cfg->n_layers * ctx->layer_stride[0];
-    // zero-fill: masked keys multiply stale values by an exact 0, which must not meet NaN or Inf bit patterns
-    ST_CREATE_CUDA(cudaMemset(ctx->pool_alloc, 0, pool_bytes));
+    // Masked keys multiply whatever the page holds by a weight of (almost) exactly 0, which must not meet NaN or Inf bit
+    // patterns: the pools start zero-filled. With ST_CFG_DEBUG_CHECKS they start filled with a large finite bf16 value
+    // instead, so that a key or value read from beyond the visible ranges shows in the rows instead of vanishing.
+    if (ctx->poison) {
+      ST_CREATE_CUDA(st::launch_fill_u16(ctx->pool_alloc, pool_bytes / 2, st::kPoisonBf16, nullptr));
+    } else {
+      ST_CREATE_CUDA(cudaMemset(ctx->pool_alloc, 0, pool_bytes));
+    }
     const size_t T = cfg->max_tokens_per_call;
     for (int s = 0; s < 2; ++s) {
       ST_CREATE_CUDA(cudaMalloc(&ctx->d_ptab[s], sizeof(int32_t) * (size_t)cfg->max_batch * ctx->ptab_stride[s]));
       ST_CREATE_CUDA(cudaMemset(ctx->d_ptab[s], 0, sizeof(int32_t) * (size_t)cfg->max_batch * ctx->ptab_stride[s]));
       ST_CREATE_CUDA(cudaMalloc(&ctx->qhat[s], T * cfg->n_q_heads * 256));
-      ST_CREATE_CUDA(cudaMalloc(&ctx->stage_q[s], T * cfg->n_q_heads * 256));
-      ST_CREATE_CUDA(cudaMalloc(&ctx->stage_k[s], T * cfg->n_kv_heads * 256));
-      ST_CREATE_CUDA(cudaMalloc(&ctx->stage_v[s], T * cfg->n_kv_heads * 256));
-      ST_CREATE_CUDA(cudaMalloc(&ctx->stage_out[s], T * cfg->n_q_heads * 512));
     }
     ST_CREATE_CUDA(cudaMalloc(&ctx->partial, sizeof(float) * st::decode_partial_floats(st::kMaxSeqPerLaunch, cfg->n_kv_heads, ctx->num_sms)));
     {
@@ -689,10 +741,20 @@ int st_reset(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq) {
     ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     ST_CUDA(ctx, cudaDeviceSynchronize());
   }
+  cudaError_t fill_err = cudaSuccess;
   auto reset_one = [&](int id) {
     SeqState &sq = ctx->seqs[id];
     for (int s = 0; s < 2; ++s) {
-      for (auto it = sq.pages[s].rbegin(); it != sq.pages[s].rend(); ++it) ctx->free_pages[s].push_back(*it);
+      for (auto it = sq.pages[s].rbegin(); it != sq.pages[s].rend(); ++it) {
+        ctx->free_pages[s].push_back(*it);
+        if (ctx->poison && !ctx->host_only) {
+          // a released page goes back to the sentinel in every layer (debug contexts only)
+          const size_t page_bytes = (size_t)ctx->cfg.n_kv_heads * st::kBlockBytes;
+          for (int layer = 0; layer < ctx->cfg.n_layers && fill_err == cudaSuccess; ++layer)
+            fill_err = st::launch_fill_u16(ctx->pool[s] + (size_t)layer * ctx->layer_stride[s] + (size_t)*it * page_bytes,
+                                           page_bytes / 2, st::kPoisonBf16, nullptr);
+        }
+      }
       sq.pages[s].clear();
     }
     sq = SeqState();
@@ -703,6 +765,8 @@ int st_reset(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq) {
     for (int i = 0; i < n_seq; ++i) reset_one(seq_ids[i]);
   }
   ctx->pend[0].active = ctx->pend[1].active = false;
+  if (fill_err != cudaSuccess) return fail(ctx, ST_ERR_CUDA, std::string("sentinel fill: ") + cudaGetErrorString(fill_err));
+  if (ctx->poison && !ctx->host_only) ST_CUDA(ctx, cudaDeviceSynchronize());
   return ST_OK;
 }
 
@@ -847,6 +911,8 @@ int st_device_status(st_ctx *ctx) {
   ST_CUDA(ctx, cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
   if (h != st::kDevOk) {
     ST_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    if (h == st::kDevBadPage)
+      return fail(ctx, ST_ERR_DEVICE_CHECK, "a page id read from a page table lies outside its pool; the access was skipped");
     return fail(ctx, ST_ERR_DEVICE_TIMEOUT, h == st::kDevTimeoutDecode    ? "a bounded wait expired in the decode kernel"
                                             : h == st::kDevTimeoutPrefill ? "a bounded wait expired in the tensor-core attention kernel"
                                                                           : "a bounded wait expired in the wait-expiry test kernel");
@@ -860,6 +926,23 @@ int st_debug_wait_expiry(st_ctx *ctx, int32_t limit_ms, void *stream) {
   if (ctx->host_only) return ST_OK;
   ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
   ST_CUDA(ctx, st::launch_wait_expiry(ctx->d_status, (uint64_t)limit_ms * 1000000ull, (cudaStream_t)stream));
+  return ST_OK;
+}
+
+int st_debug_fail_after(st_ctx *ctx, int32_t n_steps) {
+  if (!ctx || n_steps < 0) return ST_ERR_INVALID_ARG;
+  ctx->fail_countdown = n_steps;
+  return ST_OK;
+}
+
+int st_debug_corrupt_page_table(st_ctx *ctx, int32_t seq_id, int32_t which, int32_t index, int32_t page, void *stream) {
+  if (!ctx || seq_id < 0 || seq_id >= ctx->cfg.max_batch || which < 0 || which > 1) return ST_ERR_INVALID_ARG;
+  if (index < 0 || index >= ctx->ptab_stride[which]) return fail(ctx, ST_ERR_INVALID_ARG, "page table index out of range");
+  if (ctx->host_only) return ST_OK;
+  ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  ST_CUDA(ctx, cudaMemcpyAsync(ctx->d_ptab[which] + (size_t)seq_id * ctx->ptab_stride[which] + index, &page, sizeof(int32_t),
+                               cudaMemcpyHostToDevice, (cudaStream_t)stream));
+  ST_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
   return ST_OK;
 }
 

@@ -488,14 +488,17 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       for (int j = 0; j < n_max; ++j) {
         const int n_pg = min(2, n_pages - 2 * j);              // pages of this tile: 2, or 1 in an odd tail
         const uint8_t *src[2];
+        bool pages_ok = true;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const int pg = min(2 * j + h, n_pages - 1);
           const bool in_a = pg < nA;
           const int page = in_a ? p.ptab_a[(size_t)sq.slot * p.ptab_stride_a + pg]
                                 : p.ptab_b[(size_t)sq.slot * p.ptab_stride_b + (pg - nA)];
+          pages_ok = pages_ok && page_ok(page, in_a ? p.n_pages_a : p.n_pages_b, abort_flag, p.status);
           src[h] = (in_a ? p.pool_a : p.pool_b) + ((size_t)page * Hkv + kvh) * kBlockBytes;
         }
+        if (!pages_ok) break;   // nothing is copied from an address built on a bad page id
         {
           const int st = j % kKStages;
           const uint32_t use = (uint32_t)(j / kKStages);

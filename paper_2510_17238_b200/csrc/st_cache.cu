@@ -8,6 +8,8 @@
 // by more than a bf16 ulp.
 #include <string.h>
 
+#include <algorithm>
+
 #include "st_internal.h"
 
 namespace st {
@@ -55,6 +57,10 @@ __global__ void __launch_bounds__(256) st_k_rope_append(const __grid_constant__ 
   grid_dep_wait();   // the angles above need no memory; everything below reads what earlier kernels wrote
 
   const int page = p.ptab[(size_t)sq.slot * p.ptab_stride + (pos_lo >> 6)];
+  if ((unsigned)page >= (unsigned)p.n_pages) {   // block-uniform: nothing is written through a bad page id
+    if (threadIdx.x == 0) atomicExch(p.status, kDevBadPage);
+    return;
+  }
   const int Hq = p.n_q_heads, Hkv = p.n_kv_heads;
   uint8_t *page_base = p.pool + (size_t)page * Hkv * kBlockBytes;
   const int row0 = sq.q_begin + (pos_lo - sq.pos0);  // packed row of the group's first token
@@ -164,6 +170,20 @@ __global__ void st_k_wait_expiry(int32_t *status, uint64_t limit_ns) {
 
 cudaError_t launch_wait_expiry(int32_t *status, uint64_t limit_ns, cudaStream_t stream) {
   st_k_wait_expiry<<<1, 32, 0, stream>>>(status, limit_ns);
+  return cudaGetLastError();
+}
+
+__global__ void st_k_fill_u16(uint16_t *dst, size_t n, uint16_t value) {
+  // n is even and dst 4-byte aligned for every caller (whole cache blocks): two words per store
+  const uint32_t pair = (uint32_t)value | ((uint32_t)value << 16);
+  uint32_t *d = reinterpret_cast<uint32_t *>(dst);
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n / 2; i += (size_t)gridDim.x * blockDim.x) d[i] = pair;
+}
+
+cudaError_t launch_fill_u16(void *dst, size_t n, uint16_t value, cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  const size_t blocks = std::min<size_t>((n / 2 + 255) / 256, 148 * 16);
+  st_k_fill_u16<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<uint16_t *>(dst), n, value);
   return cudaGetLastError();
 }
 

@@ -46,6 +46,7 @@ constexpr int kDevOk = 0;
 constexpr int kDevTimeoutDecode = 1;
 constexpr int kDevTimeoutPrefill = 2;
 constexpr int kDevTimeoutProbe = 3;     // the wait-expiry test kernel
+constexpr int kDevBadPage = 4;          // a page id read from a page table lies outside its pool: the access was skipped
 
 // ------------------------------------------------------------------------------------------
 // Launch parameter blocks (passed by value: stream ordered, no staging buffers).
@@ -64,6 +65,8 @@ struct AppendParams {
   uint8_t *pool;                   // layer base of the pool written to
   const int32_t *ptab;             // [max_batch][ptab_stride] page ids
   int32_t ptab_stride;
+  int32_t n_pages;                 // pages of the pool: a page id outside [0, n_pages) is reported, not used
+  int32_t *status;                 // device status word
   int32_t n_seq, n_q_heads, n_kv_heads;
   double inv_freq[64];             // theta^(-2c/128), c = 0..63
   AppendSeq seq[kMaxSeqPerLaunch];
@@ -86,6 +89,7 @@ struct AttnParams {
   const uint8_t *pool_a, *pool_b;  // layer bases
   const int32_t *ptab_a, *ptab_b;
   int32_t ptab_stride_a, ptab_stride_b;
+  int32_t n_pages_a, n_pages_b;    // pages of each pool: a page id outside [0, n_pages) is reported, not used
   const __nv_bfloat16 *qhat;
   // Decode with the append fused in (q_raw != nullptr): the step's un-rotated inputs, packed [n_seq][heads][128];
   // the kernel rotates them, writes the new token into cache B and does not read qhat.
@@ -151,22 +155,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Non-blocking probe of an mbarrier phase.
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+}
+
+// Page id check of every page-table read that turns into an address: an id outside the pool is recorded in the status
+// word and the caller skips the access (no trap, no fault). One compare in one lane per 32 KiB block.
+__device__ __forceinline__ bool page_ok(int page, int n_pages, volatile int *abort_flag, int32_t *status) {
+  if ((unsigned)page < (unsigned)n_pages) return true;
+  *abort_flag = 1;
+  atomicExch(status, kDevBadPage);
+  return false;
 }
 
 // Bounded wait on an mbarrier phase. Gives up after kWaitLimitNs of wall time (or when another
@@ -193,35 +194,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
-}
-
-// The same wait for a whole converged warp, for latency-critical hand-offs: lane 0 spins on the non-blocking
-// test_wait and the result is broadcast. A thread suspended inside try_wait (or in nanosleep) was seen to notice
-// a completed phase only 400-800 cycles later, and hundreds of threads polling one mbarrier word slow each other
-// down; a single spinning lane per warp reacts within a shared-memory round trip.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                               int32_t *status, int code) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) {
-    uint64_t t0 = 0;
-    uint32_t polls = 0;
-    while (!mbar_test_wait(bar, parity)) {
-      if ((++polls & 4095u) == 0u) {
-        if (*abort_flag) { ok = 0; break; }
-        const uint64_t now = global_timer_ns();
-        if (t0 == 0) t0 = now;
-        if (now - t0 > kWaitLimitNs) {
-          *abort_flag = 1;
-          atomicExch(status, code);
-          ok = 0;
-          break;
-        }
-      }
-    }
-  }
-  ok = __shfl_sync(0xffffffffu, ok, 0);
-  __syncwarp();   // orders the other lanes' later accesses after lane 0's acquire
-  return ok != 0;
 }
 
 // One contiguous bulk copy global -> shared, completion counted in bytes on an mbarrier.

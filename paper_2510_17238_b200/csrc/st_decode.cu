@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         const bool last_of_pair = cur.t == cur.nA + cur.nB - 1;
         const int page = in_a ? p.ptab_a[(size_t)sq.slot * p.ptab_stride_a + cur.t]
                               : p.ptab_b[(size_t)sq.slot * p.ptab_stride_b + (cur.t - cur.nA)];
+        if (!page_ok(page, in_a ? p.n_pages_a : p.n_pages_b, abort_flag, p.status)) break;
         const uint8_t *src = (in_a ? p.pool_a : p.pool_b) + ((size_t)page * Hkv + cur.kvh) * kBlockBytes;
         if (!mbar_wait(smem_u32(&sm.empty[stage]), phase ^ 1u, abort_flag, p.status, kDevTimeoutDecode)) break;
         if (fused && last_of_pair) {
@@ -260,6 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sm.q_ready[slot]));     // to the consumers: the pair's queries are in place
+        if (owns_last && !page_ok(page, p.n_pages_b, abort_flag, p.status)) break;   // (warp-uniform) nothing is written
         if (owns_last) {
           uint8_t *blk = const_cast<uint8_t *>(p.pool_b) + ((size_t)page * Hkv + kvh) * kBlockBytes;
           const int tok = pos & 63;
@@ -469,6 +471,8 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
 __global__ void __launch_bounds__(128) st_k_decode_merge(const __grid_constant__ AttnParams p) {
   grid_dep_launch();
   grid_dep_wait();
+  // a decode kernel that gave up (expired wait, page id outside the pool) left partial records unwritten: merge nothing
+  if (*(volatile const int32_t *)p.status != kDevOk) return;
   const int Hkv = p.n_kv_heads, G = p.group;
   const int seq_i = blockIdx.x / p.n_q_heads, qh = blockIdx.x % p.n_q_heads;
   const int kvh = qh / G, h = qh % G;

@@ -49,7 +49,25 @@ int static_fail(char *err, int32_t cap, int code, const std::string &msg) {
 
 }  // namespace
 
-extern "C" int st_decode_attention_static(int32_t device, const void *pool_source, const void *pool_reason,
+namespace {
+
+// Makes `device` current for the duration of a call and puts the caller's device back afterwards.
+struct DeviceScope {
+  int previous = -1;
+  cudaError_t enter(int device) {
+    cudaError_t e = cudaGetDevice(&previous);
+    if (e != cudaSuccess) { previous = -1; return e; }
+    return previous == device ? cudaSuccess : cudaSetDevice(device);
+  }
+  ~DeviceScope() {
+    if (previous >= 0) cudaSetDevice(previous);
+  }
+};
+
+}  // namespace
+
+extern "C" int st_decode_attention_static(int32_t device, const void *pool_source, int64_t n_pages_source,
+                                          const void *pool_reason, int64_t n_pages_reason,
                                           const int32_t *page_table_source, int32_t table_stride_source,
                                           const int32_t *page_table_reason, int32_t table_stride_reason,
                                           const int32_t *slots, const int32_t *source_len, const int32_t *reason_len,
@@ -61,6 +79,8 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
   if (!pool_source || !pool_reason || !page_table_source || !page_table_reason || !slots || !source_len || !reason_len ||
       !q_rotated || !out)
     return static_fail(err, err_cap, ST_ERR_INVALID_ARG, "NULL argument");
+  if (n_pages_source < 1 || n_pages_reason < 1 || n_pages_source > INT32_MAX || n_pages_reason > INT32_MAX)
+    return static_fail(err, err_cap, ST_ERR_INVALID_ARG, "n_pages_source and n_pages_reason must be between 1 and 2^31 - 1");
   if (n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || n_q_heads / n_kv_heads > st::kMaxGroup)
     return static_fail(err, err_cap, ST_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads with at most 8 q heads per kv head");
   if (n_seq < 1) return static_fail(err, err_cap, ST_ERR_INVALID_ARG, "n_seq must be >= 1");
@@ -76,7 +96,8 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
       return static_fail(err, err_cap, ST_ERR_INVALID_ARG, "a length exceeds what its page table row can describe");
   }
 
-  cudaError_t e = cudaSetDevice(device);
+  DeviceScope scope;
+  cudaError_t e = scope.enter(device);
   if (e != cudaSuccess) return static_fail(err, err_cap, ST_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e));
   StaticDevice dev;
   {
@@ -105,6 +126,8 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
   p.ptab_b = page_table_reason;
   p.ptab_stride_a = table_stride_source;
   p.ptab_stride_b = table_stride_reason;
+  p.n_pages_a = (int32_t)n_pages_source;
+  p.n_pages_b = (int32_t)n_pages_reason;
   p.qhat = (const __nv_bfloat16 *)q_rotated;
   p.out = (float *)out;
   p.partial = dev.partials;
@@ -129,8 +152,25 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
   e = cudaMemsetAsync(dev.status, 0, sizeof(int32_t), s);
   if (e != cudaSuccess) return static_fail(err, err_cap, ST_ERR_CUDA, std::string("cudaMemsetAsync: ") + cudaGetErrorString(e));
   int n_launches = 0;
-  // the decode grid has at most 2 CTAs per SM; clamp so that it never exceeds the built-in capacity
-  e = st::launch_decode(p, dev.num_sms < kStaticMaxCtas / 2 ? dev.num_sms : kStaticMaxCtas / 2, s, &n_launches);
+  // the decode grid is one CTA per SM; the clamp keeps it within the built-in capacity on any device
+  e = st::launch_decode(p, dev.num_sms < kStaticMaxCtas ? dev.num_sms : kStaticMaxCtas, s, &n_launches);
   if (e != cudaSuccess) return static_fail(err, err_cap, ST_ERR_CUDA, std::string("decode launch: ") + cudaGetErrorString(e));
   return ST_OK;
+}
+
+extern "C" int st_decode_static_status(int32_t device, void *stream) {
+  if (device < 0 || device >= kStaticMaxDevices) return ST_ERR_INVALID_ARG;
+  StaticDevice dev;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    dev = g_static_device[device];
+  }
+  if (!dev.ready) return ST_ERR_INVALID_ARG;
+  DeviceScope scope;
+  if (scope.enter(device) != cudaSuccess) return ST_ERR_CUDA;
+  int32_t h = 0;   // (a stack word: the copy below allocates nothing)
+  if (cudaMemcpyAsync(&h, dev.status, sizeof(h), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
+  if (h == st::kDevOk) return ST_OK;
+  return h == st::kDevBadPage ? ST_ERR_DEVICE_CHECK : ST_ERR_DEVICE_TIMEOUT;
 }

@@ -56,6 +56,10 @@ cudaError_t launch_rope_table(const double *inv_freq, double2 *table, int n, int
 // Test surface: one warp waits (at most limit_ns) for a barrier that nothing arrives at, then records kDevTimeoutProbe.
 cudaError_t launch_wait_expiry(int32_t *status, uint64_t limit_ns, cudaStream_t stream);
 
+// Fills n 16-bit words with `value` (debug contexts: the sentinel of free pages).
+cudaError_t launch_fill_u16(void *dst, size_t n, uint16_t value, cudaStream_t stream);
+constexpr uint16_t kPoisonBf16 = 0x7149;   // bf16 0x7149 = 9.96e29: large, finite, and finite after 128-term dot products
+
 // One-time per-process function attribute set-up (dynamic shared memory opt-in).
 cudaError_t init_kernels();
 

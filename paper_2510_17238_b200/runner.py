@@ -45,8 +45,13 @@ class Plan:
 
 
 def make_plan(scheds, mode: str = "decode", lookahead: int = 1, final_chunk: int = 128,
-              explicit_units: bool = False) -> Plan:
-    """mode 'decode': reasoning tokens one by one; 'extend': one span per reasoning unit."""
+              explicit_units: bool = False, lag_units: int = 0) -> Plan:
+    """mode 'decode': reasoning tokens one by one; 'extend': one span per reasoning unit.
+
+    lag_units > 0: reasoning unit u asks for source unit min(u + lag_units, U) explicitly (lag 1 is the literal
+    reading of Eq. 2's indicator); the prefill side must then run at least lag_units + 1 units ahead."""
+    if lag_units > 0 and lookahead < lag_units + 1:
+        raise ValueError("lookahead must be at least lag_units + 1")
     B = len(scheds)
     U = max(len(s.src_unit_len) for s in scheds)
     off = np.zeros(B + 1, np.int64)
@@ -59,7 +64,8 @@ def make_plan(scheds, mode: str = "decode", lookahead: int = 1, final_chunk: int
     max_tokens = 1
     ragged = any(len(set(s.rsn_unit_len)) > 1 or s.rsn_unit_len != scheds[0].rsn_unit_len for s in scheds) or \
         any(len(s.src_unit_len) != U for s in scheds)
-    explicit = explicit_units or ragged
+    explicit = explicit_units or ragged or lag_units > 0
+    seen_unit = lambda b, u: min(u + 1 + lag_units, len(scheds[b].src_unit_len))
 
     def emit_append(u):
         nonlocal n_src, max_tokens
@@ -96,7 +102,7 @@ def make_plan(scheds, mode: str = "decode", lookahead: int = 1, final_chunk: int
         if not ids:
             return
         m = [scheds[b].rsn_unit_len[u] for b in ids]
-        vis = [u + 1] * len(ids) if explicit else None
+        vis = [seen_unit(b, u) for b in ids] if explicit else None
         if mode == "extend":
             emit_reasoning(ids, m, vis, api.ST_END_OF_UNIT, u)
             return
@@ -105,7 +111,7 @@ def make_plan(scheds, mode: str = "decode", lookahead: int = 1, final_chunk: int
         for t in range(steps):
             act = [(b, mm) for b, mm in zip(ids, m) if mm > t]
             last = uniform and t == steps - 1
-            emit_reasoning([b for b, _ in act], [1] * len(act), None if vis is None else [u + 1] * len(act),
+            emit_reasoning([b for b, _ in act], [1] * len(act), None if vis is None else [seen_unit(b, u) for b, _ in act],
                            api.ST_END_OF_UNIT if last else 0, u)
         if not uniform or steps == 0:
             # close the unit for every sequence with an empty span that only carries the flag

@@ -149,10 +149,3 @@ def qkv(index: int, sched: SeqSchedule, seq: int, layer: int = 0, seed: int = 0,
     k = _draw(seed, index, layer, seq, "k", T, w.n_kv_heads, w.head_dim, w)
     v = _draw(seed, index, layer, seq, "v", T, w.n_kv_heads, w.head_dim, w)
     return q, k, v
-
-
-def pages_needed(scheds, page_size: int = PAGE_SIZE):
-    """(source pages, reasoning pages) that hold every sequence of ``scheds`` completely."""
-    ps = sum((s.S + page_size - 1) // page_size for s in scheds)
-    pr = sum((s.R + page_size - 1) // page_size for s in scheds)
-    return ps, pr

@@ -66,6 +66,88 @@ def test_ragged_edges(hq):
         assert pu.check_cache(ctx, w, scheds, plan, flats[0]) <= 2
 
 
+def test_ragged_edges_with_sentinel_filled_pages():
+    """The ragged schedules on a debug context (ST_CFG_DEBUG_CHECKS): every free page, and so the unwritten tail of
+    every sequence's last page, holds 9.95e29 instead of zeros. A kernel that reads a key or value one token, one
+    tile or one page too far would no longer multiply it by zero quietly: the rows would leave the tolerance.
+    A second pass after st_reset runs on released pages, which are filled with the sentinel again."""
+    w = small_workload(40)
+    scheds = [
+        workloads.SeqSchedule((1, 7, 8, 63, 64, 65), (1, 0, 3, 2, 0, 5), 3),
+        workloads.SeqSchedule((255, 256, 1), (4, 0, 1), 0),
+        workloads.SeqSchedule((64, 64), (64, 1), 70),
+        workloads.SeqSchedule((130,), (0,), 2),
+    ]
+    for mode in ("decode", "extend"):
+        ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode=mode, lookahead=2, cfg_flags=api.ST_CFG_DEBUG_CHECKS)
+        pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], what=f"sentinel pages {mode}")
+        # the sentinel really is there: the token after the last one of sequence 3's source cache (130 tokens, so 62
+        # unwritten slots in its third page) reads back as the sentinel through the page table
+        ctx.reset()
+        batch2 = runner.DeviceBatch(plan, *flats[0])
+        runner.CompiledPlan(ctx, plan, [batch2]).replay()
+        torch.cuda.synchronize()
+        ctx.device_status()
+        pu.check_against_oracle(w, scheds, plan, batch2, flats[0], what=f"sentinel pages after reset {mode}")
+        ctx.close()
+
+
+def test_eq2_literal_lag_and_input_far_ahead():
+    """Two visibility variants on the GPU. (1) Eq. 2 read literally lets reasoning unit u see source unit u + 1:
+    every reasoning call names visible_units = N_EOT + 2 and the rows must equal the oracle's lag_units = 1
+    schedule. (2) Algorithm 1's "input ahead" branch: the prefill side runs three units ahead of the reasoning
+    side on workload 1, and the default visibility must still slice the source cache back to unit N_EOT + 1."""
+    w = small_workload(32)
+    scheds = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0)]
+    for mode in ("decode", "extend"):
+        _, plan, batches, flats = pu.run_plan(w, scheds, 0, mode=mode, lookahead=2, lag_units=1)
+        assert any(c.vis is not None and c.unit >= 0 and (c.vis == c.unit + 2).all() for c in plan.calls)
+        pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], what=f"lag 1 {mode}", lag_units=1)
+    w1 = workloads.WORKLOADS[1]
+    s1 = workloads.schedules(1, batch=3)
+    _, plan, batches, flats = pu.run_plan(w1, s1, 1, mode="decode", lookahead=3)
+    pu.check_against_oracle(w1, s1, plan, batches[0], flats[0], n_random=64, full_seqs=(1,), what="cfg1 lookahead 3")
+
+
+def test_page_id_outside_the_pool_is_reported_not_dereferenced():
+    """The kernels compare every page id they read with the pool's page count before they build an address from it.
+    The test overwrites one entry of the device page table with an id far outside the pool (a host-side test hook,
+    nothing on the device is broken on purpose): the next decode step reports ST_ERR_DEVICE_CHECK through the status
+    word, nothing faults, and after st_reset the context computes correct rows again."""
+    w = workloads.WORKLOADS[0]
+    scheds = workloads.schedules(0)
+    plan = runner.make_plan(scheds, mode="decode")
+    ctx = runner.make_context(w, scheds, plan)
+    flat = runner.flatten_inputs(0, scheds, layer=0)
+    dev = torch.device("cuda", 0)
+    z = lambda n, H: torch.zeros((n, H, 128), dtype=torch.bfloat16, device=dev)
+    Hq, Hkv = w.n_q_heads, w.n_kv_heads
+    for which, call in ((0, "decode"), (1, "decode"), (0, "append")):
+        # a short sound prefix: one source unit of 32 tokens and three decode steps
+        ctx.append_source_chunk(0, [0], [0, 32], z(32, Hq), z(32, Hkv), z(32, Hkv), None, api.ST_END_OF_UNIT)
+        out = torch.full((1, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
+        for _ in range(3):
+            ctx.reason_decode(0, [0], None, z(1, Hq), z(1, Hkv), z(1, Hkv), out)
+        ctx.device_status()
+        ctx.debug_corrupt_page_table(0, which, 0, 1 << 20)
+        if call == "decode":
+            ctx.reason_decode(0, [0], None, z(1, Hq), z(1, Hkv), z(1, Hkv), out)
+        else:
+            ctx.append_source_chunk(0, [0], [0, 1], z(1, Hq), z(1, Hkv), z(1, Hkv), out)
+        with pytest.raises(api.StError) as e:
+            ctx.device_status()
+        assert e.value.code == api.ST_ERR_DEVICE_CHECK
+        ctx.device_status()                                   # cleared by the read
+        ctx.reset()                                           # new appends rewrite the table entries
+        batch = runner.DeviceBatch(plan, *flat)
+        runner.CompiledPlan(ctx, plan, [batch]).replay()
+        torch.cuda.synchronize()
+        ctx.device_status()
+        pu.check_against_oracle(w, scheds, plan, batch, flat, what=f"after a bad page id in table {which}")
+        ctx.reset()
+    ctx.close()
+
+
 def test_more_sequences_than_one_launch_holds():
     """130 sequences in one call: a kernel launch carries at most 112, so every call is split into two launches."""
     w = small_workload(16)
@@ -121,50 +203,58 @@ def test_kernel_timers_sample_every_nth_decode_launch_and_leave_results_alone():
 def test_decode_steps_at_large_positions():
     """Decode steps whose token sits at reasoning positions ~69,630 (across a multiple of 1024): the append that
     runs inside the decode kernel takes cos/sin from two tables by an angle addition, and the rotated keys it
-    writes must still be the oracle's bf16(RoPE_fp64(k)) bit for bit; the rows are checked against attention
-    computed from the oracle's primitives over the cache that was read back."""
+    writes must still be the oracle's bf16(RoPE_fp64(k)) bit for bit. Everything expected comes from the oracle on
+    the raw inputs: the whole reasoning cache (the 69,629 keys the span append wrote and the 6 of the decode steps)
+    against expected_cache, and the decode rows against attention_rows."""
+    import time
     from oracle import streaming_attention as osa
-    Hq = Hkv = 8
+    Hq, Hkv = 4, 2
     S, R0, steps, theta = 64, 69_629, 6, 1.0e6
-    cfg = api.make_config(n_q_heads=Hq, n_kv_heads=Hkv, max_batch=1, n_pages_source=2, n_pages_reason=(R0 + steps) // 64 + 2,
-                          max_source_len=128, max_reason_len=R0 + steps + 64, max_tokens_per_call=8192, rope_theta=theta)
+    R = R0 + steps
+    cfg = api.make_config(n_q_heads=Hq, n_kv_heads=Hkv, max_batch=1, n_pages_source=2, n_pages_reason=R // 64 + 2,
+                          max_source_len=128, max_reason_len=R + 64, max_tokens_per_call=8192, rope_theta=theta)
     ctx = api.Context(cfg)
     dev = torch.device("cuda", 0)
     g = torch.Generator().manual_seed(7)
     draw = lambda n, H: torch.randn((n, H, 128), generator=g).to(torch.bfloat16)
     stream = torch.cuda.current_stream().cuda_stream
-    q, k, v = draw(S, Hq), draw(S, Hkv), draw(S, Hkv)
-    ctx.append_source_chunk(0, [0], [0, S], q.to(dev), k.to(dev), v.to(dev), None, api.ST_END_OF_UNIT, stream)
+    q_all, k_all, v_all = draw(S + R, Hq), draw(S + R, Hkv), draw(S + R, Hkv)     # layout [source ; reasoning]
+    ctx.append_source_chunk(0, [0], [0, S], q_all[:S].to(dev), k_all[:S].to(dev), v_all[:S].to(dev), None,
+                            api.ST_END_OF_UNIT, stream)
     done = 0
     while done < R0:                                            # cache-only spans (no attention) up to position R0
         n = min(8192, R0 - done)
-        q, k, v = draw(n, Hq), draw(n, Hkv), draw(n, Hkv)
-        ctx.reason_extend(0, [0], [0, n], [api.ST_VIS_ALL], q.to(dev), k.to(dev), v.to(dev), None, 0, stream)
+        sl = slice(S + done, S + done + n)
+        ctx.reason_extend(0, [0], [0, n], [api.ST_VIS_ALL], q_all[sl].to(dev), k_all[sl].to(dev), v_all[sl].to(dev), None, 0, stream)
         done += n
-    qs, ks, vs, outs = draw(steps, Hq), draw(steps, Hkv), draw(steps, Hkv), []
+    outs = []
     for i in range(steps):
+        sl = slice(S + R0 + i, S + R0 + i + 1)
         out = torch.full((1, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
-        ctx.reason_decode(0, [0], [api.ST_VIS_ALL], qs[i : i + 1].to(dev), ks[i : i + 1].to(dev), vs[i : i + 1].to(dev), out, 0, stream)
+        ctx.reason_decode(0, [0], [api.ST_VIS_ALL], q_all[sl].to(dev), k_all[sl].to(dev), v_all[sl].to(dev), out, 0, stream)
         outs.append(out)
     torch.cuda.synchronize()
     ctx.device_status()
     as_f64 = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).double().numpy()
-    pos = np.arange(R0, R0 + steps)
-    # the tokens the decode kernel appended
-    kg, vg = (as_f64(a) for a in ctx.debug_read_cache(0, 0, 1, R0, steps))
-    want_k = osa.round_to_bf16(osa.rope(ks.double().numpy(), pos, theta))
-    assert np.array_equal(vg, vs.double().numpy())
-    assert int((kg != want_k).sum()) <= 1 and np.abs(kg - want_k).max() <= np.abs(want_k).max() * 2.0 ** -7
-    # rows: attention over the caches as stored
-    k_src, v_src = (as_f64(a) for a in ctx.debug_read_cache(0, 0, 0, 0, S))
-    k_rsn, v_rsn = (as_f64(a) for a in ctx.debug_read_cache(0, 0, 1, 0, R0 + steps))
-    q_hat = osa.round_to_bf16(osa.rope(qs.double().numpy(), pos, theta))
+
+    t0 = time.perf_counter()
+    sched = osa.build_schedule([S], [0], R)                     # one source unit, every reasoning token final-depth
+    kd, vd = k_all.double().numpy(), v_all.double().numpy()
+    (ks_want, vs_want), (kr_want, vr_want) = osa.expected_cache(sched, kd, vd, theta)
+    # both caches as stored against the oracle's definition (at most a couple of one-ulp rounding disagreements)
+    for which, kw, vw, n in ((0, ks_want, vs_want, S), (1, kr_want, vr_want, R)):
+        kg, vg = (as_f64(a) for a in ctx.debug_read_cache(0, 0, which, 0, n))
+        assert np.array_equal(vg, vw)
+        diff = kg != kw
+        assert int(diff.sum()) <= 4, f"cache {which}: {int(diff.sum())} rotated keys differ from the oracle's"
+        assert (np.abs(kg[diff] - kw[diff]) <= np.abs(kw[diff]) * 2.0 ** -7).all()
+        if which == 1:
+            assert int(diff[R0:].sum()) <= 1                      # the six keys the decode kernel appended
+    rows = S + R0 + np.arange(steps)
+    want = osa.attention_rows(sched, q_all.double().numpy(), kd, vd, rows, theta=theta)
+    print(f"oracle: {time.perf_counter() - t0:.1f} s for both caches and {steps} rows over {S + R} keys")
     for i in range(steps):
-        keys = np.concatenate([k_src, k_rsn[: R0 + i + 1]])      # [T, H, 128]
-        vals = np.concatenate([v_src, v_rsn[: R0 + i + 1]])
-        z = np.einsum("hd,thd->ht", q_hat[i], keys) / np.sqrt(128.0)
-        want = np.einsum("ht,thd->hd", osa.softmax_rows(z), vals)
-        pu.compare(outs[i][0].cpu().numpy(), want, f"decode step at position {R0 + i}")
+        pu.compare(outs[i][0].cpu().numpy(), want[i], f"decode step at position {R0 + i}")
     ctx.close()
 
 

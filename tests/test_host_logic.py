@@ -260,3 +260,40 @@ def test_layer_protocol():
     ctx.reason_decode(1, [0], None, None, None, None, None)
     ctx.reason_decode(2, [0], None, None, None, None, None)
     assert ctx.seq_state(0)["reason_len"] == 1
+
+
+def test_a_failing_device_step_rolls_the_call_back():
+    """A CUDA failure in the middle of a call (injected on the host: the n-th device step of the call reports
+    ST_ERR_CUDA before it does anything) leaves the context as it was: pages back in the free list in their old
+    order, lengths and counters unchanged, no step pending, so that the same call can simply be issued again."""
+    steps_of_an_append = 4          # page-table update, staging, append launch, attention launch
+    for fail_at in range(1, steps_of_an_append + 1):
+        ctx = host_ctx(n_pages_source=6, n_pages_reason=4, max_batch=2)
+        ctx.append_source_chunk(0, [0], [0, 70], None, None, None, None, api.ST_END_OF_UNIT)
+        before = (ctx.pages_free(), ctx.seq_state(0), ctx.seq_state(1),
+                  ctx.debug_page_table(0, 0).tolist(), ctx.debug_page_table(1, 0).tolist())
+        ctx.debug_fail_after(fail_at)
+        rc = ctx.append_source_chunk(0, [0, 1], [0, 100, 165], None, None, None, None, api.ST_END_OF_UNIT, check=False)
+        assert rc == api.ST_ERR_CUDA and "injected" in ctx.last_error()
+        after = (ctx.pages_free(), ctx.seq_state(0), ctx.seq_state(1),
+                 ctx.debug_page_table(0, 0).tolist(), ctx.debug_page_table(1, 0).tolist())
+        assert after == before
+        # not pending: layer 0 is accepted again, takes the very same pages and commits
+        ctx.append_source_chunk(0, [0, 1], [0, 100, 165], None, None, None, None, api.ST_END_OF_UNIT)
+        assert ctx.seq_state(0) == {"source_len": 170, "reason_len": 0, "n_eos": 2, "n_eot": 0}
+        assert ctx.debug_page_table(0, 0).tolist() == [0, 1, 2] and ctx.debug_page_table(1, 0).tolist() == [3, 4]
+    # reasoning side (its first device step is the wait for the source append), and a multi-layer context: a
+    # failure at a later layer keeps the step pending at that layer, so the layer can be issued again
+    ctx = host_ctx(n_layers=2, n_pages_source=2, n_pages_reason=2, max_batch=1)
+    for layer in (0, 1):
+        ctx.append_source_chunk(layer, [0], [0, 10], None, None, None, None, api.ST_END_OF_UNIT)
+    ctx.debug_fail_after(1)
+    assert ctx.reason_decode(0, [0], None, None, None, None, None, check=False) == api.ST_ERR_CUDA
+    assert ctx.pages_free() == (1, 2) and ctx.seq_state(0)["reason_len"] == 0
+    ctx.reason_decode(0, [0], None, None, None, None, None)
+    ctx.debug_fail_after(2)
+    assert ctx.reason_decode(1, [0], None, None, None, None, None, check=False) == api.ST_ERR_CUDA
+    assert ctx.seq_state(0)["reason_len"] == 0 and ctx.pages_free() == (1, 1)
+    assert ctx.reason_decode(0, [0], None, None, None, None, None, check=False) == api.ST_ERR_STATE   # still pending
+    ctx.reason_decode(1, [0], None, None, None, None, None)
+    assert ctx.seq_state(0)["reason_len"] == 1

@@ -127,24 +127,48 @@ def rand_qkv(rng, T, Hq, Hkv, d, bf16=True):
 
 # ----------------------------------------------------------------------------- tests
 
-@pytest.mark.parametrize("n,m,f,Hq,Hkv,d", [
-    ([2, 3, 1], [1, 2, 2], 2, 2, 1, 4),
-    ([1, 1, 1, 1], [1, 1, 1, 1], 0, 2, 2, 8),
-    ([3, 2], [0, 2], 1, 4, 2, 4),
-    ([4], [3], 0, 1, 1, 8),
+@pytest.mark.parametrize("n,m,f,Hq,Hkv,d,row_block", [
+    ([2, 3, 1], [1, 2, 2], 2, 2, 1, 4, 256),
+    ([1, 1, 1, 1], [1, 1, 1, 1], 0, 2, 2, 8, 256),
+    ([3, 2], [0, 2], 1, 4, 2, 4, 256),
+    ([4], [3], 0, 1, 1, 8, 256),
+    # the oracle's loop over blocks of rows, with several blocks and a ragged last one: 11 rows in blocks of 3,
+    # 8 rows in blocks of 1 and 7 rows in blocks of 4
+    ([2, 3, 1], [1, 2, 2], 2, 2, 1, 4, 3),
+    ([1, 1, 1, 1], [1, 1, 1, 1], 0, 2, 2, 8, 1),
+    ([4], [3], 0, 1, 1, 8, 4),
 ])
-def test_brute_force_tiny(n, m, f, Hq, Hkv, d):
+def test_brute_force_tiny(n, m, f, Hq, Hkv, d, row_block):
     rng = np.random.default_rng(11)
     sched = osa.build_schedule(n, m, f)
     q, k, v = rand_qkv(rng, sched.S + sched.R, Hq, Hkv, d)
     want = brute_force(n, m, f, q, k, v, Hq, Hkv, THETA)
-    got = osa.attention_rows(sched, q, k, v, np.arange(sched.S + sched.R), theta=THETA, round_rotated=False)
+    got = osa.attention_rows(sched, q, k, v, np.arange(sched.S + sched.R), theta=THETA, round_rotated=False,
+                             row_block=row_block)
     assert np.abs(got - want).max() < 1e-12
     # with the two bf16 rounding points (rounded through torch, not the oracle's routine)
     want_r = brute_force(n, m, f, q, k, v, Hq, Hkv, THETA, round_fn=bf16_via_torch)
-    got_r = osa.attention_rows(sched, q, k, v, np.arange(sched.S + sched.R), theta=THETA, round_rotated=True)
+    got_r = osa.attention_rows(sched, q, k, v, np.arange(sched.S + sched.R), theta=THETA, round_rotated=True,
+                               row_block=row_block)
     assert np.abs(got_r - want_r).max() < 1e-12
     assert np.abs(got_r - got).max() > 1e-6      # the rounding is really applied
+
+
+def test_row_subsets_in_any_order_across_blocks():
+    """Rows may be listed in any order, repeated, and spread over several row blocks: every listed row equals the
+    scalar loops' row (the GPU parity tests hand the oracle sampled row lists longer than one block)."""
+    rng = np.random.default_rng(12)
+    n, m, f, Hq, Hkv, d = [3, 1, 4], [2, 0, 3], 2, 4, 2, 8
+    sched = osa.build_schedule(n, m, f)
+    T = sched.S + sched.R
+    q, k, v = rand_qkv(rng, T, Hq, Hkv, d)
+    want = brute_force(n, m, f, q, k, v, Hq, Hkv, THETA)
+    rows = np.array([T - 1, 0, 9, 9, 3, 12, 1, 8, 14, 2, 5])
+    for blk in (2, 5, 256):
+        got, probs = osa.attention_rows(sched, q, k, v, rows, theta=THETA, round_rotated=False, row_block=blk,
+                                        return_probs=True)
+        assert np.abs(got - want[rows]).max() < 1e-12
+        assert np.abs(probs.sum(-1) - 1).max() < 1e-12
 
 
 def sdpa_causal(qr, kr, v, G, scale):

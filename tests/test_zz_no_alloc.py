@@ -5,7 +5,9 @@ owns the GPU, or they cannot take the device-wide stall of cudaMalloc), so this 
 split-K workspace in an array built into the library. The GPU test drives a small batch through the
 regular calls and, for two decode steps in a row, computes the same rows again through the
 allocation-free entry point: it must reproduce st_reason_decode within the parity tolerance of the
-other tests (in fact bit for bit, since the same kernels run on the same split plan).
+other tests (in fact bit for bit, since the same kernels run on the same split plan), and the fp64
+oracle's rows within the same tolerance. The page tables of this call are the caller's, so the test
+also hands it a table with a page id outside the pool and expects an error status instead of a fault.
 
 This file sorts last on purpose, so a run that stops at the first failure has run everything else.
 """
@@ -22,21 +24,26 @@ REL_L2_TOL = 5e-3
 
 def test_static_entry_rejects_oversized_calls_with_a_message():
     # validation happens before any CUDA call, so this part needs no GPU
-    dummy = np.zeros(4, np.int32)
+    call = lambda **kw: api.decode_attention_static(**{**dict(
+        device=0, pool_source=1024, n_pages_source=4, pool_reason=1024, n_pages_reason=4, page_table_source=1024,
+        table_stride_source=4, page_table_reason=1024, table_stride_reason=4, slots=[0], source_len=[1], reason_len=[1],
+        q_rotated=1024, out=1024, n_q_heads=32, n_kv_heads=8, check=False), **kw})
     n = 65                                                  # 65 sequences x 8 kv heads > 512 pairs
-    rc, msg = api.decode_attention_static(0, 1024, 1024, 1024, 4, 1024, 4, [0] * n, [1] * n, [1] * n, 1024, 1024,
-                                          32, 8, check=False)
+    rc, msg = call(slots=[0] * n, source_len=[1] * n, reason_len=[1] * n)
     assert rc == api.ST_ERR_INVALID_ARG and "at most" in msg and "512" in msg
-    rc, msg = api.decode_attention_static(0, 1024, 1024, 1024, 4, 1024, 4, [0] * 113, [1] * 113, [1] * 113, 1024, 1024,
-                                          8, 1, check=False)
+    rc, msg = call(slots=[0] * 113, source_len=[1] * 113, reason_len=[1] * 113, n_q_heads=8, n_kv_heads=1)
     assert rc == api.ST_ERR_INVALID_ARG and "112" in msg
-    rc, msg = api.decode_attention_static(0, 1024, 1024, 1024, 4, 1024, 4, [0], [1], [0], 1024, 1024, 32, 8, check=False)
+    rc, msg = call(reason_len=[0])
     assert rc == api.ST_ERR_INVALID_ARG and "reason_len" in msg
-    rc, msg = api.decode_attention_static(0, 1024, 1024, 1024, 1, 1024, 4, [0], [65], [1], 1024, 1024, 32, 8, check=False)
+    rc, msg = call(table_stride_source=1, source_len=[65])
     assert rc == api.ST_ERR_INVALID_ARG and "page table" in msg
-    rc, msg = api.decode_attention_static(0, None, 1024, 1024, 4, 1024, 4, [0], [1], [1], 1024, 1024, 32, 8, check=False)
+    rc, msg = call(pool_source=None)
     assert rc == api.ST_ERR_INVALID_ARG
-    del dummy
+    rc, msg = call(n_pages_reason=0)
+    assert rc == api.ST_ERR_INVALID_ARG and "n_pages" in msg
+    # the status reader refuses a device on which no such call has been made (and bad ordinals)
+    assert api.decode_static_status(63) == api.ST_ERR_INVALID_ARG
+    assert api.decode_static_status(-1) == api.ST_ERR_INVALID_ARG
 
 
 @pytest.mark.gpu
@@ -99,15 +106,40 @@ def test_static_entry_matches_reason_decode_two_calls_in_a_row():
         got = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
         torch.cuda.synchronize()
         free_before = torch.cuda.mem_get_info()[0]
-        api.decode_attention_static(0, pool_source, pool_reason, tab_s, stride_s, tab_r, stride_r, ids,
+        api.decode_attention_static(0, pool_source, ps, pool_reason, pr, tab_s, stride_s, tab_r, stride_r, ids,
                                     [scheds[b].S for b in ids], [st["reason_len"] for st in state], q_rot, got,
                                     Hq, Hkv, stream=stream)
         torch.cuda.synchronize()
+        assert api.decode_static_status(0, stream) == api.ST_OK
         if step == 1:
             # (the very first call may make the driver load the library image that holds the workspace)
             assert torch.cuda.mem_get_info()[0] >= free_before - (1 << 20), "the call must not allocate device memory"
         g, r = got.double().cpu().numpy(), want.double().cpu().numpy()
         assert not np.isnan(g).any()
         assert np.abs(g - r).max() <= MAX_ABS_TOL and np.linalg.norm(g - r) / np.linalg.norm(r) <= REL_L2_TOL
+        # and against the fp64 oracle on the raw inputs, row by row
+        for b, s in enumerate(scheds):
+            o = osa.build_schedule(s.src_unit_len, s.rsn_unit_len, s.final_len)
+            qd, kd, vd = (t.double().numpy() for t in tensors[b])
+            ref = osa.attention_rows(o, qd, kd, vd, [rows[b]], theta=w.rope_theta)[0]
+            assert np.abs(g[b] - ref).max() <= MAX_ABS_TOL
+            assert np.linalg.norm(g[b] - ref) / np.linalg.norm(ref) <= REL_L2_TOL
+
+    # A page id outside the pool in the caller's table: the kernel must not build an address from it. The call
+    # still returns ST_OK (it only queues work); the status reader reports the failed check, nothing faults, and
+    # the rows of the sequence -- long enough to be split over several CTAs, so that only the merge kernel would
+    # write them -- stay untouched. The next call with a sound table is correct again.
+    bad_s = tab_s.clone()
+    bad_s[0, 3] = ps + 1000
+    got_bad = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
+    args = (ids, [scheds[b].S for b in ids], [st["reason_len"] for st in state], q_rot)
+    api.decode_attention_static(0, pool_source, ps, pool_reason, pr, bad_s, stride_s, tab_r, stride_r, *args, got_bad,
+                                Hq, Hkv, stream=stream)
+    assert api.decode_static_status(0, stream) == api.ST_ERR_DEVICE_CHECK
+    assert torch.isnan(got_bad[0]).all(), "rows of the sequence with the bad page id must not be written"
+    api.decode_attention_static(0, pool_source, ps, pool_reason, pr, tab_s, stride_s, tab_r, stride_r, *args, got_bad,
+                                Hq, Hkv, stream=stream)
+    assert api.decode_static_status(0, stream) == api.ST_OK
+    assert torch.equal(got_bad, got)
     ctx.device_status()
     ctx.close()
