@@ -65,6 +65,13 @@ extern "C" {
                                       that a key or value read from beyond the visible ranges -- which the
                                       kernels would otherwise multiply by a weight of zero without a trace --
                                       shows up in the rows. The kernels' page-id checks are always on.     */
+#define ST_CFG_PRECISE_P       4u  /* chunk prefill and reasoning spans carry the softmax weights into the
+                                      weights-times-values product as two bf16 terms (16 significant bits)
+                                      instead of one (8 bits). One term bounds a row's error by about 2^-9
+                                      times the largest |v| the row mixes: within 1e-2 for values of order 1,
+                                      not for values of a few tens (outlier channels). The second term costs
+                                      one more tensor-core product per key tile. Decode steps always use two
+                                      terms (free there).                                                   */
 /* per-call flags */
 #define ST_END_OF_UNIT         1u  /* source side: this chunk completes a source unit (N_EOS += 1);
                                       reasoning side: the unit's boundary token was produced (N_EOT += 1) */

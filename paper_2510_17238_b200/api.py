@@ -20,7 +20,7 @@ lib = C.CDLL(_LIB_PATH)
 
 ST_OK, ST_ERR_INVALID_ARG, ST_ERR_OOM_PAGES, ST_ERR_NOT_READY = 0, -1, -2, -3
 ST_ERR_STATE, ST_ERR_CUDA, ST_ERR_DEVICE_TIMEOUT, ST_ERR_DEVICE_CHECK = -4, -5, -6, -7
-ST_CFG_HOST_ONLY, ST_CFG_DEBUG_CHECKS = 1, 2
+ST_CFG_HOST_ONLY, ST_CFG_DEBUG_CHECKS, ST_CFG_PRECISE_P = 1, 2, 4
 ST_END_OF_UNIT, ST_REFERENCE_KERNELS, ST_IO_HOST = 1, 2, 4
 ST_VIS_DEFAULT, ST_VIS_ALL = -1, -2
 

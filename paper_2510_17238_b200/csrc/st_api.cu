@@ -75,6 +75,12 @@ struct st_ctx {
 
   std::vector<EventRec> events;
   uint64_t serial = 0;
+  // Events per source append are recorded only once a reasoning-side call has come in on another stream than the
+  // appends (an event between two kernels serialises them completely, which would keep consecutive appends from
+  // overlapping). Until then one catch-all event, recorded when such a call first needs it, covers all appends so far.
+  bool cross_stream = false;
+  cudaStream_t last_src_stream = nullptr;
+  EventRec catch_all;
   Pending pend[2];
 
   // kernel timing (benchmarks): event pairs in flight and a pool of spare events
@@ -87,6 +93,7 @@ struct st_ctx {
   std::vector<int32_t> meta_pos, meta_vis_src, meta_vis_rsn;
   std::string err;
   int64_t launches = 0;
+  bool precise_p = false;        // ST_CFG_PRECISE_P: two-term probabilities in the tensor-core attention kernel
   bool poison = false;           // ST_CFG_DEBUG_CHECKS: free pages hold a large finite sentinel instead of zeros
   int fail_countdown = 0;        // test hook: the n-th internal device step from now reports ST_ERR_CUDA
 };
@@ -141,6 +148,7 @@ void release_device(st_ctx *ctx) {
   cudaDeviceSynchronize();
   for (auto &e : ctx->events)
     if (e.ev) cudaEventDestroy(e.ev);
+  if (ctx->catch_all.ev) cudaEventDestroy(ctx->catch_all.ev);
   for (auto &t : ctx->timed) { cudaEventDestroy(t.t0); cudaEventDestroy(t.t1); }
   for (auto &e : ctx->spare_events) cudaEventDestroy(e);
   for (int s = 0; s < 2; ++s) {
@@ -283,18 +291,30 @@ int wait_for_append(st_ctx *ctx, uint64_t serial, cudaStream_t stream) {
   if (int rc = injected_failure(ctx, "stream wait")) return rc;
   if (ctx->host_only || serial == 0) return ST_OK;
   EventRec &rec = ctx->events[serial % kEventRing];
-  if (rec.serial != serial) {
+  if (rec.serial == serial) {
+    if (rec.stream != stream) ST_CUDA(ctx, cudaStreamWaitEvent(stream, rec.ev, 0));
+    return ST_OK;
+  }
+  if (rec.serial > serial) {
     // the event slot was recycled by a newer append: source appends are stream-ordered, so the
     // newest recorded event of the ring covers the one we need
     uint64_t best = 0;
     EventRec *newest = nullptr;
     for (auto &e : ctx->events)
       if (e.serial > best) { best = e.serial; newest = &e; }
-    if (!newest) return ST_OK;
-    if (newest->stream != stream) ST_CUDA(ctx, cudaStreamWaitEvent(stream, newest->ev, 0));
+    if (newest && newest->stream != stream) ST_CUDA(ctx, cudaStreamWaitEvent(stream, newest->ev, 0));
     return ST_OK;
   }
-  if (rec.stream != stream) ST_CUDA(ctx, cudaStreamWaitEvent(stream, rec.ev, 0));
+  // no event was recorded for that append (all calls came on one stream so far)
+  if (ctx->last_src_stream == stream) return ST_OK;   // same stream: stream order is enough
+  ctx->cross_stream = true;                           // from now on every append records its event
+  if (ctx->catch_all.serial < serial) {
+    if (!ctx->catch_all.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&ctx->catch_all.ev, cudaEventDisableTiming));
+    ST_CUDA(ctx, cudaEventRecord(ctx->catch_all.ev, ctx->last_src_stream));
+    ctx->catch_all.stream = ctx->last_src_stream;
+    ctx->catch_all.serial = ctx->serial;              // every append submitted so far
+  }
+  if (ctx->catch_all.stream != stream) ST_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->catch_all.ev, 0));
   return ST_OK;
 }
 
@@ -424,6 +444,7 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
   p->n_kv_heads = ctx->cfg.n_kv_heads;
   p->group = ctx->group;
   p->scale_log2 = ctx->scale_log2;
+  memcpy(p->inv_freq, ctx->inv_freq, sizeof(p->inv_freq));
   p->total_work = p->work_per_cta = p->n_cta = 0;
 }
 
@@ -431,7 +452,7 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
 // `fused`: non-null for a decode step whose append runs inside the decode kernel (the call's un-rotated q/k/v).
 int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
                   const std::vector<int32_t> &vis_tokens, float *out, uint32_t flags, cudaStream_t stream,
-                  const IoPtrs *fused) {
+                  const IoPtrs &io, bool fused) {
   if (int rc = injected_failure(ctx, "attention launch")) return rc;
   if (ctx->host_only || !out) return ST_OK;
   const int side = kind == 0 ? 0 : 1;
@@ -442,11 +463,13 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
     st::AttnParams ap;
     fill_attn_common(ctx, side, layer, out, &ap);
     if (fused) {
-      ap.q_raw = fused->q;
-      ap.k_raw = fused->k;
-      ap.v_raw = fused->v;
+      ap.q_raw = io.q;
+      ap.k_raw = io.k;
+      ap.v_raw = io.v;
       ap.rope_hi = ctx->rope_hi;
       ap.rope_lo = ctx->rope_lo;
+    } else if (kind != 1 && !(flags & ST_REFERENCE_KERNELS)) {
+      ap.q_raw = io.q;   // the tensor-core kernel rotates its query rows itself
     }
     int n_used = 0;
     for (int i = 0; i < ns; ++i) {
@@ -484,7 +507,7 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
     } else if (kind == 1) {
       ST_CUDA(ctx, st::launch_decode(ap, ctx->num_sms, stream, &nl, t0, t1));
     } else {
-      ST_CUDA(ctx, st::launch_attn_tc(ap, ctx->num_sms, stream, &nl, t0, t1));
+      ST_CUDA(ctx, st::launch_attn_tc(ap, ctx->precise_p, ctx->num_sms, stream, &nl, t0, t1));
     }
     ctx->launches += nl;
   }
@@ -561,17 +584,25 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     // A decode step's append (one token per sequence) runs inside the decode kernel: the step is then two kernels
     // instead of three. Cache-only calls and the cross-check kernels keep the separate append.
     const bool fuse_append = kind == 1 && io.out != nullptr && !(flags & ST_REFERENCE_KERNELS) && !ctx->host_only;
-    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, io, io.out != nullptr, stream))) return r;
-    if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, io.out, flags, stream,
-                           fuse_append ? &io : nullptr))) return r;
+    // Rotated queries go to scratch only for the kernels that read them there: the simple cross-check kernels and a
+    // decode step whose append is not fused, and the tensor-core kernel's two-term variant (which wants the fp64
+    // rotation). The one-term tensor-core kernel rotates its own.
+    const bool want_qhat = io.out != nullptr && ((flags & ST_REFERENCE_KERNELS) || kind == 1 || ctx->precise_p);
+    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, io, want_qhat, stream))) return r;
+    if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, io.out, flags, stream, io, fuse_append))) return r;
     if ((r = unstage_output(ctx, side, flags, total, out, stream, io))) return r;
     if (layer == ctx->cfg.n_layers - 1 && kind == 0 && !ctx->host_only) {
-      // the event later reasoning-side calls wait for
+      // the event later reasoning-side calls on another stream wait for
       EventRec &rec = ctx->events[(ctx->serial + 1) % kEventRing];
-      if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
-      ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
-      rec.stream = stream;
-      rec.serial = ctx->serial + 1;
+      if (ctx->cross_stream) {
+        if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
+        ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
+        rec.stream = stream;
+        rec.serial = ctx->serial + 1;
+      } else {
+        rec.serial = 0;   // none recorded: wait_for_append falls back to the catch-all event
+      }
+      ctx->last_src_stream = stream;
     }
     return ST_OK;
   };
@@ -637,7 +668,7 @@ int st_create(const st_config *cfg, st_ctx **out) {
   if (!out) { g_create_error = "out is NULL"; return ST_ERR_INVALID_ARG; }
   *out = nullptr;
   if (!config_ok(cfg, &why)) { g_create_error = why; return ST_ERR_INVALID_ARG; }
-  if (cfg->flags & ~(ST_CFG_HOST_ONLY | ST_CFG_DEBUG_CHECKS)) { g_create_error = "unknown config flag"; return ST_ERR_INVALID_ARG; }
+  if (cfg->flags & ~(ST_CFG_HOST_ONLY | ST_CFG_DEBUG_CHECKS | ST_CFG_PRECISE_P)) { g_create_error = "unknown config flag"; return ST_ERR_INVALID_ARG; }
   const uint64_t pool_bytes = st_pool_bytes(cfg);
   if (cfg->pool_base && (cfg->pool_bytes < pool_bytes || ((uintptr_t)cfg->pool_base & 1023))) {
     g_create_error = "pool_base must be 1024-byte aligned and hold st_pool_bytes() bytes";
@@ -647,6 +678,7 @@ int st_create(const st_config *cfg, st_ctx **out) {
   ctx->cfg = *cfg;
   ctx->host_only = (cfg->flags & ST_CFG_HOST_ONLY) != 0;
   ctx->poison = (cfg->flags & ST_CFG_DEBUG_CHECKS) != 0;
+  ctx->precise_p = (cfg->flags & ST_CFG_PRECISE_P) != 0;
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / sqrt((double)cfg->head_dim);
   ctx->scale_log2 = (float)(scale * 1.4426950408889634);
@@ -765,6 +797,7 @@ int st_reset(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq) {
     for (int i = 0; i < n_seq; ++i) reset_one(seq_ids[i]);
   }
   ctx->pend[0].active = ctx->pend[1].active = false;
+  if (n_seq == 0) ctx->cross_stream = false;   // a full reset (which waited for the device) starts in single-stream mode again
   if (fill_err != cudaSuccess) return fail(ctx, ST_ERR_CUDA, std::string("sentinel fill: ") + cudaGetErrorString(fill_err));
   if (ctx->poison && !ctx->host_only) ST_CUDA(ctx, cudaDeviceSynchronize());
   return ST_OK;

@@ -22,8 +22,9 @@
 // Operands. The cache block layout in HBM already is the 128-byte-swizzled K-major shared-memory operand
 // format, so panels are used as landed: the two pages' K panels of one channel half are placed one after the
 // other and form a 128-key operand; every V^T panel (channels x 64 keys) serves four 16-key steps of P V.
-// Q tiles are copied into the same format by the softmax warps with asynchronous 16-byte copies (whole rows per
-// copy instruction).
+// Q tiles are copied into the same format by the softmax warps with asynchronous 16-byte copies (whole rows per copy
+// instruction) from the caller's un-rotated queries, and rotated in place at their position ids (the two-term variant
+// takes them rotated from the append kernel's scratch instead).
 // Tensor memory (512 columns): S[t] (128 fp32 columns per M-tile) and O[t] (128 columns per M-tile).
 // Schedule per M-tile and key tile j (the MMA pipe executes in issue order, which is what the aliasing relies on):
 //   the softmax warps work S(j) off as two 64-key online-softmax steps (one cache page each);
@@ -48,7 +49,8 @@ namespace st {
 
 namespace {
 
-constexpr int kKStages = 2;                 // K ring depth (32 KiB per stage: 128 keys x 128 channels)
+constexpr int kKStagesFast = 2;             // K ring depth (32 KiB per stage: 128 keys x 128 channels); the two-term
+                                            // variant gives its second stage to the low-order P of the second key half
 constexpr int kVStages = 2;                 // V ring depth (32 KiB per stage: two V^T page panels)
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kThreads = 320;               // 8 softmax warps, producer, MMA issuer
@@ -59,12 +61,16 @@ constexpr int kKStageBytes = 32768;         // 2 channel halves x 128 keys x 128
 constexpr int kVStageBytes = 32768;         // 2 pages x 128 channels x 128 B (64 keys)
 constexpr int kHalfPanel = 16384;           // one channel half of a 128-row tile / one V^T page panel
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
-constexpr uint32_t kPolyPairs = 0x92u;      // of every 8 score pairs, those whose bit is set take the polynomial exp2
+#ifndef ST_ATTN_POLY_PAIRS
+#define ST_ATTN_POLY_PAIRS 0x92u
+#endif
+constexpr uint32_t kPolyPairs = ST_ATTN_POLY_PAIRS;   // of every 8 score pairs, those whose bit is set take the polynomial exp2
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + 2 * kQTileBytes;
-constexpr int kOffV = kOffK + kKStages * kKStageBytes;
+constexpr int kOffP1Lo = kOffK + kKStageBytes;            // two-term variant only: low-order P of the second key half, per M-tile
+constexpr int kOffV = kOffK + kKStagesFast * kKStageBytes;
 constexpr int kOffP1 = kOffV + kVStages * kVStageBytes;   // P of the second key half, per M-tile: 128 rows x 64 keys bf16
 constexpr int kP1Bytes = 16384;
 constexpr int kOffBar = kOffP1 + 2 * kP1Bytes;
@@ -73,8 +79,8 @@ static_assert(kSmemBytes + 1024 <= 232448, "shared memory budget of one CTA");
 
 struct Barriers {
   uint64_t q_full[2];
-  uint64_t k_full[kKStages];
-  uint64_t k_empty[kKStages];
+  uint64_t k_full[kKStagesFast];
+  uint64_t k_empty[kKStagesFast];
   uint64_t v_full[kVStages];
   uint64_t v_empty[kVStages];
   uint64_t s_full[2];     // S[t](j) complete
@@ -209,6 +215,13 @@ __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
         "l"(reinterpret_cast<const uint64_t &>(c)));
   return d;
 }
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+  float2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;"
+      : "=l"(reinterpret_cast<uint64_t &>(d))
+      : "l"(reinterpret_cast<const uint64_t &>(a)), "l"(reinterpret_cast<const uint64_t &>(b)));
+  return d;
+}
 __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
   float2 d;
   asm("add.rn.f32x2 %0, %1, %2;"
@@ -233,6 +246,16 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23)),
                      __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23)));
 }
+__device__ __forceinline__ float sin_approx(float x) {
+  float y;
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float cos_approx(float x) {
+  float y;
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 // acc_lo += low bf16 of pk, acc_hi += high bf16 of pk (fp32 accumulation of bf16 terms)
 __device__ __forceinline__ void add_bf16x2(float &acc_lo, float &acc_hi, uint32_t pk) {
   asm("{\n.reg .b16 lo, hi;\n"
@@ -245,7 +268,12 @@ __device__ __forceinline__ void add_bf16x2(float &acc_lo, float &acc_hi, uint32_
 
 }  // namespace
 
+// kPrecise: the probabilities enter P V as two bf16 terms (p = hi + lo, 16 significant bits) instead of one. One bf16
+// term bounds a row's error by about 2^-9 times the largest |v| it mixes, which leaves the 1e-2 tolerance when values
+// reach a few tens (outlier channels); the second term costs one more P V product per key tile.
+template <bool kPrecise>
 __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constant__ AttnParams p) {
+  constexpr int kKStages = kPrecise ? 1 : kKStagesFast;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Barriers &bar = *reinterpret_cast<Barriers *>(smem + kOffBar);
@@ -302,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar.tmem_base;
-  grid_dep_wait();   // set-up above touches no global memory; the rotated queries and the cache pages come from earlier kernels
+  grid_dep_wait();   // set-up above touches no global memory; the cache pages come from earlier kernels
 
   if (warp < 8) {
     // =========================================================== softmax + epilogue warps
@@ -315,26 +343,93 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       const uint32_t s_base = lane_addr + kColS + (uint32_t)(t * 128);
       const uint32_t o_addr = lane_addr + kColO + (uint32_t)(t * 128);
 
-      // ---- Q tile into the swizzled K-major layout, by asynchronous 16-byte copies. The tile's 128 threads copy
-      // it 8 rows at a time: 16 lanes take the 16 chunks of one row, so every copy instruction reads whole
+      // ---- Q tile into the swizzled K-major operand layout, by asynchronous 16-byte copies. The tile's 128 threads
+      // copy it 8 rows at a time: 16 lanes take the 16 chunks of one row, so every copy instruction reads whole
       // 256-byte rows; rows past the end of the sequence are zero-filled (source size 0, nothing is read).
+      // Two-term variant: the rows come rotated from the append kernel's scratch (fp64 rotation, exactly the rounding
+      // bf16(RoPE(q)); needed when channels of large magnitude make a one-ulp difference in a rotated query visible).
+      // One-term variant: the rows come un-rotated from the caller's buffer and are rotated in place below.
+      uint8_t *q_tile = smem + kOffQ + t * kQTileBytes;
       {
+        const __nv_bfloat16 *q_src = kPrecise ? p.qhat : p.q_raw;
         const int c = r_local & 15;                          // chunk of the row
-        const uint32_t q_smem = smem_u32(smem + kOffQ + t * kQTileBytes);
+        const uint32_t q_smem = smem_u32(q_tile);
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const int rr = i * 8 + (r_local >> 4);              // row of the tile
           const int grow = row0 + t * kRowsPerTile + rr;
           const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
           const bool in = grow < packed_rows;
-          const __nv_bfloat16 *src = in ? p.qhat + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + c * 8 : p.qhat;
+          const __nv_bfloat16 *src = in ? q_src + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + c * 8 : q_src;
           cp_async16(q_smem + (c >> 3) * kHalfPanel + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src, in ? 16u : 0u);
         }
         cp_async_wait_all();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bar.q_full[t]));
       }
+      if constexpr (!kPrecise) {
+        // Rotation at the streaming position ids (position of token tk of the call = tokens already in the cache + tk),
+        // in place. One work item = (token, 16-byte chunk c and its partner c + 8, i.e. channels 8c..8c+7 and 64+8c..):
+        // its cos/sin are computed once and serve the G query heads of the token. The angle pos * inv_freq is formed
+        // and reduced to a fraction of a turn in fp64 (an fp32 angle would be off by a bf16 ulp of the result at
+        // positions of a few 10^4); sine, cosine and the rotation run in fp32, whose error (1e-6 of |q|) is three
+        // orders below the bf16 rounding that follows: about one rotated element in 10^4 lands on the other side of
+        // a rounding boundary than the fp64 rotation would put it.
+        tile_sync(t);                                          // every thread's copies have landed
+        const int r_lo = row0 + t * kRowsPerTile;              // first packed row of the tile
+        const int r_end = min(r_lo + kRowsPerTile, packed_rows);
+        const int tok_lo = div_g(r_lo), tok_hi = div_g(r_end - 1);
+        const int n_items = (tok_hi - tok_lo + 1) * 8;
+        for (int it = r_local; it < n_items; it += kRowsPerTile) {
+          const int tk = tok_lo + (it >> 3), c = it & 7;
+          float cs[8], sn[8];
+          const double pos = (double)(sq.b_base + tk);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const double turns = pos * p.inv_freq[8 * c + e] * 0.15915494309189535;   // angle / 2 pi
+            const float r = (float)(turns - rint(turns)) * 6.2831853071795865f;       // in [-pi, pi]
+            sn[e] = sin_approx(r);
+            cs[e] = cos_approx(r);
+          }
+          // all rows of the item are read before the first is written back (the compiler cannot move a shared-memory
+          // load over a store of the row before it, and with two warps per scheduler nothing else hides that latency)
+          uint4 lo_raw[kMaxGroup], hi_raw[kMaxGroup];
+#pragma unroll
+          for (int g = 0; g < kMaxGroup; ++g) {
+            const int rr = tk * G + g - r_lo;
+            if (g < G && rr >= 0 && rr < r_end - r_lo) {
+              const uint8_t *ptr = q_tile + rr * 128 + ((c ^ (rr & 7)) << 4);
+              lo_raw[g] = *reinterpret_cast<const uint4 *>(ptr);
+              hi_raw[g] = *reinterpret_cast<const uint4 *>(ptr + kHalfPanel);
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < kMaxGroup; ++g) {
+            const int rr = tk * G + g - r_lo;
+            if (g < G && rr >= 0 && rr < r_end - r_lo) {
+              const uint32_t *lo_w = reinterpret_cast<const uint32_t *>(&lo_raw[g]);
+              const uint32_t *hi_w = reinterpret_cast<const uint32_t *>(&hi_raw[g]);
+              uint32_t lo_out[4], hi_out[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // two channels per word: x = channels 8c+2e, 8c+2e+1, y = their partners 64 channels on
+                const float2 x = make_float2(__uint_as_float(lo_w[e] << 16), __uint_as_float(lo_w[e] & 0xffff0000u));
+                const float2 y = make_float2(__uint_as_float(hi_w[e] << 16), __uint_as_float(hi_w[e] & 0xffff0000u));
+                const float2 c2 = make_float2(cs[2 * e], cs[2 * e + 1]), s2 = make_float2(sn[2 * e], sn[2 * e + 1]);
+                const float2 ns2 = make_float2(-sn[2 * e], -sn[2 * e + 1]);
+                const float2 lo_r = ffma2(x, c2, fmul2(y, ns2));          // x cos - y sin
+                const float2 hi_r = ffma2(y, c2, fmul2(x, s2));           // y cos + x sin
+                lo_out[e] = cvt_bf16x2(lo_r.x, lo_r.y);
+                hi_out[e] = cvt_bf16x2(hi_r.x, hi_r.y);
+              }
+              uint8_t *ptr = q_tile + rr * 128 + ((c ^ (rr & 7)) << 4);
+              *reinterpret_cast<uint4 *>(ptr) = make_uint4(lo_out[0], lo_out[1], lo_out[2], lo_out[3]);
+              *reinterpret_cast<uint4 *>(ptr + kHalfPanel) = make_uint4(hi_out[0], hi_out[1], hi_out[2], hi_out[3]);
+            }
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar.q_full[t]));
 
       const float c_log2 = p.scale_log2;
       float m_ref = -INFINITY, l_sum = 0.f;                   // m_ref in scaled (log2) units
@@ -390,6 +485,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
           uint32_t packed[32];
+          uint32_t packed_lo[kPrecise ? 32 : 1];
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             // The special-function unit does 16 exp2 per clock and SM, exactly the rate at which the tensor core
@@ -406,7 +502,14 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
             }
             const uint32_t pk = cvt_bf16x2(e0, e1);
             packed[c] = pk;
-            add_bf16x2(acc[2 * (c & 1)], acc[2 * (c & 1) + 1], pk);   // sum what the tensor core will use
+            if constexpr (kPrecise) {
+              // second term: what the first left over; hi + lo carries 16 bits of p, so the row sum takes p itself
+              packed_lo[c] = cvt_bf16x2(e0 - __uint_as_float(pk << 16), e1 - __uint_as_float(pk & 0xffff0000u));
+              acc[2 * (c & 1)] += e0;
+              acc[2 * (c & 1) + 1] += e1;
+            } else {
+              add_bf16x2(acc[2 * (c & 1)], acc[2 * (c & 1) + 1], pk);   // sum what the tensor core will use
+            }
           }
           l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
 
@@ -416,6 +519,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           const bool rescale = (j > 0 || h > 0) && __any_sync(0xffffffffu, grow);
           if (h == 0) {
             tmem_st32(s_addr, packed);                          // P: 64 keys as 32 packed columns, over the scores
+            if constexpr (kPrecise) tmem_st32(s_addr + 32, packed_lo);   // (columns 32-63 of the half were read above)
             if (rescale && !mbar_wait(smem_u32(&bar.p1_free[t]), (j - 1) & 1, abort_flag, p.status, kDevTimeoutPrefill)) { ok = false; break; }
           } else {
             if (j > 0 && !mbar_wait(smem_u32(&bar.p1_free[t]), (j - 1) & 1, abort_flag, p.status, kDevTimeoutPrefill)) { ok = false; break; }
@@ -423,6 +527,13 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
             for (int c8 = 0; c8 < 8; ++c8)                      // K-major operand layout, 128-byte swizzle
               *reinterpret_cast<uint4 *>(p1_row + ((c8 ^ (r_local & 7)) << 4)) =
                   make_uint4(packed[c8 * 4], packed[c8 * 4 + 1], packed[c8 * 4 + 2], packed[c8 * 4 + 3]);
+            if constexpr (kPrecise) {
+              uint8_t *lo_row = smem + kOffP1Lo + t * kP1Bytes + r_local * 128;
+#pragma unroll
+              for (int c8 = 0; c8 < 8; ++c8)
+                *reinterpret_cast<uint4 *>(lo_row + ((c8 ^ (r_local & 7)) << 4)) =
+                    make_uint4(packed_lo[c8 * 4], packed_lo[c8 * 4 + 1], packed_lo[c8 * 4 + 2], packed_lo[c8 * 4 + 3]);
+            }
             fence_proxy_async_smem();
             if (rescale && !mbar_wait(smem_u32(&bar.pv0_done[t]), j & 1, abort_flag, p.status, kDevTimeoutPrefill)) { ok = false; break; }
           }
@@ -553,11 +664,22 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
           tc_mma_ts(d, pa + ks * 8, vd + (uint64_t)((ks * 32) >> 4), idesc, (j > 0 || ks > 0) ? 1u : 0u, issue);
+        if constexpr (kPrecise) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            tc_mma_ts(d, pa + 32 + ks * 8, vd + (uint64_t)((ks * 32) >> 4), idesc, 1u, issue);
+        }
       } else {
         const uint64_t pd = make_desc(p1_addr + t * kP1Bytes);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
           tc_mma_ss(d, pd + (uint64_t)((ks * 32) >> 4), vd + (uint64_t)((ks * 32) >> 4), idesc, 1u, issue);
+        if constexpr (kPrecise) {
+          const uint64_t pl = make_desc(smem_u32(smem + kOffP1Lo) + t * kP1Bytes);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            tc_mma_ss(d, pl + (uint64_t)((ks * 32) >> 4), vd + (uint64_t)((ks * 32) >> 4), idesc, 1u, issue);
+        }
       }
     };
 
@@ -632,12 +754,14 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
 }
 
 cudaError_t init_attn_tc_kernels() {
-  return cudaFuncSetAttribute(st_k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
+  cudaError_t e = cudaFuncSetAttribute(st_k_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(st_k_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
 }
 
 int attn_tc_rows_per_cta() { return kRowsPerCta; }
 
-cudaError_t launch_attn_tc(AttnParams &p, int num_sms, cudaStream_t stream, int *n_launches, cudaEvent_t t0,
+cudaError_t launch_attn_tc(AttnParams &p, bool precise, int num_sms, cudaStream_t stream, int *n_launches, cudaEvent_t t0,
                            cudaEvent_t t1) {
   (void)num_sms;
   *n_launches = 0;
@@ -650,7 +774,8 @@ cudaError_t launch_attn_tc(AttnParams &p, int num_sms, cudaStream_t stream, int 
   p.total_work = total;
   p.n_cta = total;
   if (t0) cudaEventRecord(t0, stream);
-  cudaError_t e = launch_dependent(st_k_attn_tc, dim3(total), dim3(kThreads), kSmemBytes + 1024, stream, p);
+  cudaError_t e = launch_dependent(precise ? st_k_attn_tc<true> : st_k_attn_tc<false>, dim3(total), dim3(kThreads),
+                                   kSmemBytes + 1024, stream, p);
   if (e != cudaSuccess) return e;
   if (t1) cudaEventRecord(t1, stream);
   *n_launches = 1;

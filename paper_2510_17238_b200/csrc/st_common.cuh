@@ -91,8 +91,9 @@ struct AttnParams {
   int32_t ptab_stride_a, ptab_stride_b;
   int32_t n_pages_a, n_pages_b;    // pages of each pool: a page id outside [0, n_pages) is reported, not used
   const __nv_bfloat16 *qhat;
-  // Decode with the append fused in (q_raw != nullptr): the step's un-rotated inputs, packed [n_seq][heads][128];
-  // the kernel rotates them, writes the new token into cache B and does not read qhat.
+  // Un-rotated inputs of the call, packed [tokens][heads][128]. Decode with the append fused in (q_raw != nullptr):
+  // the kernel rotates q and k, writes the new token into cache B and does not read qhat. Tensor-core kernel: q_raw
+  // only (always set); it rotates the rows of its Q tiles while staging them and never reads qhat.
   const __nv_bfloat16 *q_raw, *k_raw, *v_raw;
   float *out;                      // [rows][n_q_heads][128]
   float *partial;                  // split-K workspace (decode)
@@ -102,6 +103,7 @@ struct AttnParams {
   int32_t work_per_cta;            // decode: tiles per CTA
   int32_t n_cta;
   float scale_log2;                // softmax scale * log2(e)
+  double inv_freq[64];             // theta^(-2c/128): the tensor-core kernel rotates its queries itself (from q_raw)
   // decode with the append fused in: (cos, sin) of k * 1024 * inv_freq[c] and of j * inv_freq[c], j < 1024, as [.][64]
   const double2 *rope_hi, *rope_lo;
   AttnSeq seq[kMaxSeqPerLaunch];

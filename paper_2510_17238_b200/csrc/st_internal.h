@@ -23,7 +23,8 @@ cudaError_t launch_decode(AttnParams &p, int num_sms, cudaStream_t stream, int *
 size_t decode_partial_floats(int n_seq_per_launch, int n_kv_heads, int num_sms);
 
 // Multi-row attention on tensor cores (chunk prefill and reasoning spans).
-cudaError_t launch_attn_tc(AttnParams &p, int num_sms, cudaStream_t stream, int *n_launches,
+// precise: probabilities as two bf16 terms (one more P V product per key tile), for values of large magnitude.
+cudaError_t launch_attn_tc(AttnParams &p, bool precise, int num_sms, cudaStream_t stream, int *n_launches,
                            cudaEvent_t t0 = nullptr, cudaEvent_t t1 = nullptr);
 int attn_tc_rows_per_cta();
 

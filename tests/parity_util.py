@@ -41,9 +41,13 @@ def compare(got, want, what=""):
     got = np.asarray(got, dtype=np.float64)
     want = np.asarray(want, dtype=np.float64)
     assert not np.isnan(got).any(), f"{what}: NaN in the GPU output (row never written?)"
-    max_abs = float(np.abs(got - want).max())
+    err = np.abs(got - want)
+    max_abs = float(err.max())
     rel_l2 = float(np.linalg.norm(got - want) / np.linalg.norm(want))
-    assert max_abs <= MAX_ABS_TOL and rel_l2 <= REL_L2_TOL, f"{what}: max_abs={max_abs:.3e} rel_l2={rel_l2:.3e}"
+    at = tuple(int(i) for i in np.unravel_index(int(err.argmax()), err.shape))
+    assert max_abs <= MAX_ABS_TOL and rel_l2 <= REL_L2_TOL, (
+        f"{what}: max_abs={max_abs:.3e} rel_l2={rel_l2:.3e}; worst element at index {at}: got {got[at]:.6f}, "
+        f"want {want[at]:.6f}")
     return max_abs, rel_l2
 
 

@@ -92,6 +92,26 @@ def test_ragged_edges_with_sentinel_filled_pages():
         ctx.close()
 
 
+@pytest.mark.parametrize("hq", [8, 32, 40])
+def test_two_term_probabilities_on_outlier_channels(hq):
+    """ST_CFG_PRECISE_P (probabilities as two bf16 terms in chunk prefill and spans) on ragged schedules whose
+    Q, K and V carry 2 % of their (head, channel) pairs multiplied by 8: unit lengths straddle pages and tiles,
+    sequences end on odd page counts, and every row must stay within the tolerance."""
+    w = workloads.Workload(0, f"outliers-{hq}q", hq, 8, 1, outlier_frac=0.02, outlier_mult=8.0)
+    scheds = [
+        workloads.SeqSchedule((1, 7, 8, 63, 64, 65), (1, 0, 3, 2, 0, 5), 3),
+        workloads.SeqSchedule((255, 256, 1), (4, 0, 1), 0),
+        workloads.SeqSchedule((300, 212), (64, 1), 70),
+        workloads.SeqSchedule((130,), (0,), 2),
+    ]
+    for mode in ("decode", "extend"):
+        ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode=mode, lookahead=2, cfg_flags=api.ST_CFG_PRECISE_P)
+        worst = pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], what=f"two-term P hq={hq} {mode}")
+        assert worst[0] <= 5e-3, f"two-term probabilities should leave a wide margin, got {worst}"
+        assert pu.check_cache(ctx, w, scheds, plan, flats[0]) <= 2
+        ctx.close()
+
+
 def test_eq2_literal_lag_and_input_far_ahead():
     """Two visibility variants on the GPU. (1) Eq. 2 read literally lets reasoning unit u see source unit u + 1:
     every reasoning call names visible_units = N_EOT + 2 and the rows must equal the oracle's lag_units = 1
