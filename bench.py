@@ -38,6 +38,9 @@ import torch
 # DRAM bytes per algorithmic byte of st_k_decode, from an ncu capture of the small decode case (--profile-case decode:
 # 272.8 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.0177
+# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill); None until the counters of the
+# kernel as it stands have been taken.
+PREFILL_DRAM_PER_ALGORITHMIC_BYTE = None
 
 METRIC = "reasoning-decode tok/s per layer (chunk prefill concurrent on a second stream)"
 UNIT = "tok/s"
@@ -58,6 +61,10 @@ def parse_args():
                     help="side measurement: reasoning units and the final stage teacher-forced as spans "
                          "(st_reason_extend) on one stream; prints its own JSON line")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the compact measurements of workloads 4 and 3 that the default run appends as per_config")
+    ap.add_argument("--side-layers", type=int, default=4,
+                    help="layers of workload 3's 36-layer stack that the per_config measurement runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--oracle-rows", type=int, default=0, help="rows per oracle sample (0 = sized for ~15 s)")
     ap.add_argument("--profile-case", default=None, choices=["decode", "prefill"],
@@ -277,6 +284,124 @@ def whole_job_tokens_per_s(tokens_per_rank, ms_max, steps, world):
     return world * tokens_per_rank * steps / (ms_max / 1e3)
 
 
+def config_dict(w, scheds, layers, world):
+    """The `config` object of a JSON line: the same keys for the CUDA arm and the reference arm."""
+    kv_bytes = sum(s.S + s.R for s in scheds) * 2 * w.n_kv_heads * w.head_dim * 2 * layers
+    in_bytes = sum(s.S + s.R for s in scheds) * (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim * 2
+    return {"workload": w.name, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
+            "batch_per_gpu": len(scheds), "source_tokens": scheds[0].S, "reasoning_tokens": scheds[0].R, "layers": layers,
+            "page_size": 64, "streams": 2, "parallelism": f"replicas x{world} (sequences sharded, no collective)",
+            "l2": ("KV working set %.2f GiB and %.1f GB of inputs against a 126 MB L2: every step streams more than L2 "
+                   "holds; no flush" % (kv_bytes / 2**30, in_bytes / 1e9)) if kv_bytes > 2 * 126e6 else
+                  ("KV working set %.1f MB fits in L2: launch-latency-bound configuration, no flush" % (kv_bytes / 1e6))}
+
+
+def prefill_algorithmic_bytes(scheds, w):
+    """Bytes the chunk-prefill attention kernel must move in one pass: per append call and sequence the K/V of the
+    prefix and the chunk once (4096 B per token), the chunk's queries in (bf16) and its rows out (fp32)."""
+    total = 0
+    for s in scheds:
+        p = 0
+        for n in s.src_unit_len:
+            total += (p + n) * 2 * w.n_kv_heads * w.head_dim * 2 + n * w.n_q_heads * w.head_dim * (2 + 4)
+            p += n
+    return total
+
+
+def measure_prefill_alone(ctx, compiled, api, reps):
+    """Chunk prefill with no decode stream beside it. Returns (bracketed launches, their summed ms, wall ms of one
+    appends-only pass with nothing between the kernels): the first is the tensor-core kernel's own time (events around
+    every launch), the second the time of the whole append chain (page-table update, K/V append, attention)."""
+    append_only = (api.lib.st_append_source_chunk,)
+    ctx.reset()
+    compiled.replay(kinds=append_only)                       # warm-up
+    torch.cuda.synchronize()
+    ctx.kernel_timing_enable(True)
+    for _ in range(reps):
+        ctx.reset()
+        compiled.replay(kinds=append_only)
+    n, ms = ctx.kernel_timing_read(1)
+    ctx.kernel_timing_enable(False)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream = torch.cuda.current_stream()
+    chain = []
+    for _ in range(reps):
+        ctx.reset()
+        torch.cuda.synchronize()
+        # the appends run on the plan's source stream: bracket them there
+        compiled.src_stream.wait_stream(stream)
+        e0.record(compiled.src_stream)
+        compiled.replay(kinds=append_only)
+        e1.record(compiled.src_stream)
+        torch.cuda.synchronize()
+        chain.append(e0.elapsed_time(e1))
+    ctx.device_status()
+    return n, ms / reps, min(chain)
+
+
+def measure_side_config(index, args, local_rank, layers=None):
+    """Compact measurement of another workload for the `per_config` list: one timed pass of the whole plan on two
+    streams after three warm-up passes (decode tokens per second, decode kernel against HBM), and chunk prefill
+    alone (tensor-core kernel against the bf16 peak). Workload 3 runs a stated subset of its 36 layers."""
+    from paper_2510_17238_b200 import api, runner, workloads
+    w = workloads.WORKLOADS[index]
+    scheds = workloads.schedules(index)
+    L = w.n_layers if layers is None else min(layers, w.n_layers)
+    cfg_flags = api.ST_CFG_PRECISE_P if w.outlier_frac > 0 else 0   # as in the parity tests of that workload
+    plan = runner.make_plan(scheds, mode="decode", lookahead=1)
+    ctx = runner.make_context(w, scheds, plan, n_layers=L, device=local_rank, flags=cfg_flags)
+    batch = runner.DeviceBatch(plan, *gen_inputs(index, scheds))
+    s_src, s_rsn = torch.cuda.Stream(), torch.cuda.Stream()
+    compiled = runner.CompiledPlan(ctx, plan, [batch] * L, s_src, s_rsn)
+    for _ in range(3):
+        ctx.reset()
+        compiled.replay()
+    torch.cuda.synchronize()
+    ctx.device_status()
+    period = max(1, args.time_every)
+    ctx.kernel_timing_enable(period)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s_rsn)
+    s_src.wait_event(e0)
+    ctx.reset()
+    compiled.replay()
+    s_rsn.wait_stream(s_src)
+    e1.record(s_rsn)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    n_dec, ms_dec = ctx.kernel_timing_read(0)
+    ctx.kernel_timing_read(1)
+    ctx.kernel_timing_enable(False)
+    ctx.device_status()
+    peaks = measured_peaks()
+    dec_call_bytes = decode_algorithmic_bytes(plan, scheds, w)
+    timed_idx = (np.arange(n_dec, dtype=np.int64) * period) % max(len(dec_call_bytes) * L, 1)
+    dec_bytes_timed = float(dec_call_bytes[timed_idx // L].sum()) if n_dec else 0.0
+    dec_gbs = dec_bytes_timed / (ms_dec / 1e3) / 1e9 if n_dec and ms_dec > 0 else 0.0
+    n_pre, ms_pre, ms_chain = measure_prefill_alone(ctx, compiled, api, reps=2)
+    flops = prefill_algorithmic_flops(scheds, w) * L
+    tflops = flops / (ms_pre / 1e3) / 1e12 if ms_pre > 0 else 0.0
+    out = {"workload": w.name, "layers_run": L, "layers_of_workload": w.n_layers, "two_term_probabilities": bool(cfg_flags),
+           "warmup_passes": 3, "timed_passes": 1, "ms_per_pass": ms,
+           "decode_tok_s": sum(s.R for s in scheds) * L / (ms / 1e3),
+           "decode": {"kernel": "st_k_decode", "bound": "hbm", "achieved": dec_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                      "frac": dec_gbs / peaks["hbm_gbs"], "avg_launch_us": 1e3 * ms_dec / max(n_dec, 1), "launches_timed": n_dec,
+                      "algorithmic_bytes_per_launch": dec_bytes_timed / max(n_dec, 1)},
+           "prefill": {"kernel": "st_k_attn_tc", "bound": "tensor", "achieved": tflops, "unit": "TFLOP/s",
+                       "peak": peaks["bf16_tflops"], "frac": tflops / peaks["bf16_tflops"], "launches_per_pass": n_pre // 2,
+                       "kernel_ms_per_pass": ms_pre, "append_chain_ms_per_pass": ms_chain,
+                       "append_chain_tflops": flops / (ms_chain / 1e3) / 1e12,
+                       "prefill_tok_s_chain": sum(s.S for s in scheds) * L / (ms_chain / 1e3)},
+           "of": peaks["source"], "clocks": clocks}
+    ctx.close()
+    del batch, compiled
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_reference(args, w, scheds, rank, world):
     """--impl reference: the oracle on the host cores, bounded sample per step."""
     if rank != 0:
@@ -292,8 +417,7 @@ def run_reference(args, w, scheds, rank, world):
         "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(v[1] for v in vals), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
-                   "batch": len(scheds), "source_tokens": scheds[0].S, "reasoning_tokens": scheds[0].R},
+        "config": config_dict(w, scheds, w.n_layers, max(args.gpus, 1)),
         "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -431,18 +555,8 @@ def main():
 
     # ---- chunk prefill alone: the same appends with no decode stream beside them, so that the tensor-core
     # kernel's own rate is seen (in the concurrent pass its launches share the SMs with the decode kernel)
-    append_only = (api.lib.st_append_source_chunk,)
-    ctx.reset()
-    compiled.replay(kinds=append_only)
-    torch.cuda.synchronize()
-    ctx.kernel_timing_enable(True)
     solo_reps = 5
-    for _ in range(solo_reps):
-        ctx.reset()
-        compiled.replay(kinds=append_only)
-    n_pre_solo, ms_pre_solo = ctx.kernel_timing_read(1)
-    ctx.kernel_timing_enable(False)
-    ctx.device_status()
+    n_pre_solo, ms_pre_solo, ms_chain = measure_prefill_alone(ctx, compiled, api, solo_reps)
 
     B = len(scheds)
     rsn_tokens = sum(s.R for s in scheds)
@@ -450,8 +564,6 @@ def main():
     sec_per_step = ms / 1e3 / args.steps
     value = whole_job_tokens_per_s(rsn_tokens * L, ms, args.steps, world)   # per layer: token-layers per second
 
-    kv_bytes = sum(s.S + s.R for s in scheds) * 2 * w.n_kv_heads * w.head_dim * 2 * L
-    in_bytes = sum(s.S + s.R for s in scheds) * (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim * 2
     peaks = measured_peaks()
     dec_call_bytes = decode_algorithmic_bytes(plan, scheds, w)
     dec_launches = len(dec_call_bytes)                    # decode launches of one layer in one pass
@@ -475,14 +587,26 @@ def main():
                 "algorithmic_bytes_per_launch": dec_bytes_per_launch,
                 "timed": "every %d-th launch, its own bytes over its own time" % period,
                 "frac_of_nominal_8TBs": dec_gbs / 8000.0}
-    solo_tflops = pre_flops * solo_reps / (ms_pre_solo / 1e3) / 1e12 if n_pre_solo and ms_pre_solo > 0 else 0.0
+    solo_tflops = pre_flops / (ms_pre_solo / 1e3) / 1e12 if n_pre_solo and ms_pre_solo > 0 else 0.0
+    pre_bytes = prefill_algorithmic_bytes(scheds, w) * L
     roofline_prefill = {"bound": "tensor", "kernel": "st_k_attn_tc (chunk prefill)", "achieved": solo_tflops,
                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": solo_tflops / peaks["bf16_tflops"],
                         "of": peaks["source"] + " (burst: kernel timed alone, appends only, no decode stream)",
                         "frac_of_sustained": solo_tflops / peaks["bf16_tflops_sustained"],
                         "frac_of_nominal_2250": solo_tflops / 2250.0,
-                        "launches": n_pre_solo, "total_ms_per_pass": ms_pre_solo / solo_reps,
-                        "algorithmic_flops_per_pass": pre_flops, "traffic": None,
+                        "launches": n_pre_solo, "total_ms_per_pass": ms_pre_solo,
+                        "algorithmic_flops_per_pass": pre_flops,
+                        "traffic": PREFILL_DRAM_PER_ALGORITHMIC_BYTE * pre_bytes / max(n_pre_solo // solo_reps, 1)
+                        if PREFILL_DRAM_PER_ALGORITHMIC_BYTE else None,
+                        "traffic_how": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the small prefill case "
+                                       "(--profile-case prefill) per algorithmic byte (K/V of prefix and chunk once, queries "
+                                       "in, rows out), times the average algorithmic bytes of a launch of this pass",
+                        "algorithmic_bytes_per_launch": pre_bytes / max(n_pre_solo // solo_reps, 1),
+                        "append_chain": {"achieved": pre_flops / (ms_chain / 1e3) / 1e12, "ms_per_pass": ms_chain,
+                                         "what": "the same flops over the wall time of an appends-only pass with nothing "
+                                                 "between the kernels: page-table update, K/V append and attention of "
+                                                 "every call back to back",
+                                         "prefill_tok_s": world * src_tokens * L / (ms_chain / 1e3)},
                         "concurrent_with_decode": {"achieved": pre_tflops, "launches": n_pre,
                                                    "total_ms_per_step": ms_pre / args.steps}}
 
@@ -490,12 +614,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
-                   "batch_per_gpu": B, "source_tokens": scheds[0].S, "reasoning_tokens": scheds[0].R, "layers": L,
-                   "page_size": 64, "streams": 2, "parallelism": f"replicas x{world} (sequences sharded, no collective)",
-                   "l2": ("KV working set %.2f GiB and %.1f GB of inputs against a 126 MB L2: every step streams more than L2 "
-                          "holds; no flush" % (kv_bytes / 2**30, in_bytes / 1e9)) if kv_bytes > 2 * 126e6 else
-                         ("KV working set %.1f MB fits in L2: launch-latency-bound configuration, no flush" % (kv_bytes / 1e6))},
+        "config": config_dict(w, scheds, L, world),
         "clocks": clocks, "gpu_launches": int(gpu_launches),
         "decode_kernel_tok_s": (world * rsn_tokens / (dec_call_bytes.sum() / (dec_gbs * 1e9))) if dec_gbs else None,
         "prefill_kernel_tok_s": world * src_tokens * L * args.steps / (ms_pre / 1e3) if ms_pre else None,
@@ -518,6 +637,14 @@ def main():
                               "through device staging; a decode step (under 1 MiB) is read and written in place by its "
                               "kernels, every byte crossing the bus once inside the timed region"}
         del host_batch, cp_host
+
+    # ---- the other two configurations whose rooflines mean something (N = 1 only: keeps the scaling runs short)
+    if rank == 0 and world == 1 and args.config == 2 and not args.no_per_config:
+        del batch, compiled
+        ctx.close()
+        torch.cuda.empty_cache()
+        line["per_config"] = [measure_side_config(4, args, local_rank),
+                              measure_side_config(3, args, local_rank, layers=args.side_layers)]
 
     # ---- the oracle on the host cores (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -231,6 +231,7 @@ class CompiledPlan:
         self.plan = plan
         self.keep = []
         self.items = []
+        self.src_stream = stream_src if stream_src is not None else torch.cuda.current_stream()
         L = len(batches)
         s_src = stream_src.cuda_stream if stream_src is not None else torch.cuda.current_stream().cuda_stream
         s_rsn = stream_rsn.cuda_stream if stream_rsn is not None else s_src
