@@ -63,14 +63,30 @@ class Schedule:
     rsn_unit: np.ndarray      # [R] int32, unit of reasoning token r (U+1 = final depth)
 
 
-def build_schedule(src_unit_len, rsn_unit_len, final_len=0, lag_units=0) -> Schedule:
-    """Eq. 1 / Algorithm 1 (visibility) and the streaming position encoding.
+POSITION_MODES = ("streaming", "concatenated", "unit_aligned")
+
+
+def build_schedule(src_unit_len, rsn_unit_len, final_len=0, lag_units=0, position_mode="streaming") -> Schedule:
+    """Eq. 1 / Algorithm 1 (visibility) and the position ids (Section 3.2).
 
     Reasoning unit ``u`` is produced while ``N_EOS == N_EOT + 1 == u``, i.e. when
     exactly the first ``u`` source units are in the (sliced) source cache, so its
     tokens see the source prefix ``P_u``. ``lag_units`` shifts that to
     ``P_{min(u + lag, U)}``.
+
+    ``position_mode`` (source tokens always count from zero):
+
+    * ``"streaming"``: the streaming position encoding -- reasoning tokens count from
+      zero on a counter of their own (the method's encoding);
+    * ``"concatenated"``: the original RoPE ids that Section 3.2 starts from -- the
+      reasoning token with index ``t`` gets ``T + t``, ``T`` the input length (the
+      "RoPE" rows of the batch-setting comparison);
+    * ``"unit_aligned"``: a variant of this build, not the paper's: the ``i``-th token
+      of reasoning unit ``u`` gets ``P_{u-1} + i``, i.e. every reasoning unit restarts at
+      the position where its source unit starts; final-depth tokens get ``S + i``.
     """
+    if position_mode not in POSITION_MODES:
+        raise ValueError(f"position_mode must be one of {POSITION_MODES}")
     n = np.asarray(src_unit_len, dtype=np.int64).reshape(-1)
     m = np.asarray(rsn_unit_len, dtype=np.int64).reshape(-1)
     if n.shape != m.shape:
@@ -87,8 +103,21 @@ def build_schedule(src_unit_len, rsn_unit_len, final_len=0, lag_units=0) -> Sche
     pos = np.empty(S + R, dtype=np.int32)
     for j in range(S):          # source counter starts at zero
         pos[j] = j
-    for r in range(R):          # reasoning counter starts at zero too
-        pos[S + r] = r
+    if position_mode == "streaming":
+        for r in range(R):      # reasoning counter starts at zero too
+            pos[S + r] = r
+    elif position_mode == "concatenated":
+        for r in range(R):      # one counter over [input ; reasoning]
+            pos[S + r] = S + r
+    else:
+        r = 0
+        for u in range(1, U + 1):
+            for i in range(int(m[u - 1])):
+                pos[S + r] = P[u - 1] + i
+                r += 1
+        for i in range(int(final_len)):
+            pos[S + r] = S + i
+            r += 1
 
     vis = np.empty(R, dtype=np.int32)
     unit = np.empty(R, dtype=np.int32)

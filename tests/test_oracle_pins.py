@@ -213,6 +213,45 @@ def test_everything_visible_is_causal_over_concatenation():
     assert np.abs(got0[-f:] - want[-f:]).max() < 1e-12                # final-depth rows agree
 
 
+def test_concatenated_ids_with_everything_visible_is_the_batch_route():
+    """Original RoPE ids (reasoning token t at T + t, Section 3.2) with every reasoning token seeing the whole
+    input is ordinary causal attention over [input ; reasoning] with ordinary position ids 0 .. T+R-1: the single
+    cache "batch" route, computed here by torch's library routine."""
+    rng = np.random.default_rng(16)
+    n, m, f = [4, 6, 2], [3, 1, 5], 4
+    Hq, Hkv, d = 4, 2, 16
+    sched = osa.build_schedule(n, m, f, lag_units=len(n), position_mode="concatenated")
+    T = sched.S + sched.R
+    assert sched.pos_ids.tolist() == list(range(T))
+    q, k, v = rand_qkv(rng, T, Hq, Hkv, d)
+    got = osa.attention_rows(sched, q, k, v, np.arange(T), theta=THETA, round_rotated=False)
+    pos = np.arange(T)
+    want = sdpa_causal(complex_rope(q, pos, THETA), complex_rope(k, pos, THETA), v, Hq // Hkv, 1 / math.sqrt(d))
+    assert np.abs(got - want).max() < 1e-12
+    # the streaming ids give different reasoning rows on the same mask, and the same source rows
+    got_s = osa.attention_rows(osa.build_schedule(n, m, f, lag_units=len(n)), q, k, v, np.arange(T), theta=THETA,
+                               round_rotated=False)
+    assert np.abs(got_s[: sched.S] - want[: sched.S]).max() < 1e-12
+    assert np.abs(got_s[sched.S :] - want[sched.S :]).max() > 1e-4
+
+
+def test_position_modes_closed_form():
+    n, m, f = [3, 1, 4], [2, 0, 3], 2
+    S = sum(n)
+    s0 = osa.build_schedule(n, m, f)
+    s1 = osa.build_schedule(n, m, f, position_mode="concatenated")
+    s2 = osa.build_schedule(n, m, f, position_mode="unit_aligned")
+    for s in (s0, s1, s2):
+        assert s.pos_ids[:S].tolist() == list(range(S))                 # the input always counts from zero
+        assert np.array_equal(s.vis_len, s0.vis_len)                    # positions do not touch visibility
+    assert s0.pos_ids[S:].tolist() == [0, 1, 2, 3, 4, 5, 6]
+    assert s1.pos_ids[S:].tolist() == [8, 9, 10, 11, 12, 13, 14]        # T + t
+    # unit 1 starts at P_0 = 0, unit 3 at P_2 = 4, the final stage at S = 8
+    assert s2.pos_ids[S:].tolist() == [0, 1, 4, 5, 6, 8, 9]
+    with pytest.raises(ValueError):
+        osa.build_schedule(n, m, f, position_mode="other")
+
+
 def test_softmax_rows():
     rng = np.random.default_rng(7)
     n, m, f = [3, 4, 2], [2, 3, 1], 3
