@@ -83,6 +83,18 @@ extern "C" {
                                       write the rows directly in host memory. Either way the buffers belong
                                       to the call until the work queued on `stream` has completed            */
 
+/* st_config.position_mode */
+#define ST_POS_STREAMING       0   /* Section 3.2, streaming position encoding: the reasoning cache counts its
+                                      tokens from zero on a counter of its own (the method's encoding)      */
+#define ST_POS_CONCATENATED    1   /* the original RoPE ids Section 3.2 starts from: reasoning token t gets
+                                      T + t, T = tokens in the source cache when the sequence's first
+                                      reasoning token is appended (the whole input in the batch setting, where
+                                      the paper compares the two encodings)                                  */
+#define ST_POS_UNIT_ALIGNED    2   /* variant of this library, not the paper's: the i-th token of reasoning
+                                      unit u gets P_{u-1} + i (the unit restarts where its source unit starts);
+                                      tokens decoded with ST_VIS_ALL (final depth) get S + i, S = source
+                                      tokens at the first such call                                          */
+
 /* visible_units values */
 #define ST_VIS_DEFAULT        -1   /* Algorithm 1: unit N_EOT + 1                                         */
 #define ST_VIS_ALL            -2   /* everything appended so far (final-depth reasoning, Eq. 1 last term) */
@@ -108,6 +120,9 @@ typedef struct st_config {
   double   rope_theta;             /* RoPE base, e.g. 1e6                                                 */
   float    softmax_scale;          /* 0 = 1/sqrt(head_dim)                                                */
   uint32_t flags;                  /* ST_CFG_*                                                            */
+  int32_t  position_mode;          /* ST_POS_*: position ids of reasoning tokens (source tokens always count
+                                      from zero)                                                          */
+  int32_t  reserved;               /* must be 0                                                           */
 } st_config;
 
 /* Bytes of device memory the two page pools need: n_layers * (n_pages_source + n_pages_reason) *

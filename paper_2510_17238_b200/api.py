@@ -23,6 +23,7 @@ ST_ERR_STATE, ST_ERR_CUDA, ST_ERR_DEVICE_TIMEOUT, ST_ERR_DEVICE_CHECK = -4, -5, 
 ST_CFG_HOST_ONLY, ST_CFG_DEBUG_CHECKS, ST_CFG_PRECISE_P = 1, 2, 4
 ST_END_OF_UNIT, ST_REFERENCE_KERNELS, ST_IO_HOST = 1, 2, 4
 ST_VIS_DEFAULT, ST_VIS_ALL = -1, -2
+ST_POS_STREAMING, ST_POS_CONCATENATED, ST_POS_UNIT_ALIGNED = 0, 1, 2
 
 ERROR_NAMES = {0: "ST_OK", -1: "ST_ERR_INVALID_ARG", -2: "ST_ERR_OOM_PAGES", -3: "ST_ERR_NOT_READY",
                -4: "ST_ERR_STATE", -5: "ST_ERR_CUDA", -6: "ST_ERR_DEVICE_TIMEOUT", -7: "ST_ERR_DEVICE_CHECK"}
@@ -37,6 +38,7 @@ class st_config(C.Structure):
         ("max_tokens_per_call", C.c_int32), ("device", C.c_int32),
         ("pool_base", C.c_void_p), ("pool_bytes", C.c_uint64),
         ("rope_theta", C.c_double), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
+        ("position_mode", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -110,10 +112,10 @@ def st_pool_bytes(cfg: st_config) -> int:
 
 def make_config(n_layers=1, n_q_heads=16, n_kv_heads=8, max_batch=1, n_pages_source=0, n_pages_reason=0,
                 max_source_len=0, max_reason_len=0, max_tokens_per_call=1, device=0, pool_base=None, pool_bytes=0,
-                rope_theta=1.0e6, softmax_scale=0.0, flags=0) -> st_config:
+                rope_theta=1.0e6, softmax_scale=0.0, flags=0, position_mode=0) -> st_config:
     return st_config(n_layers, n_q_heads, n_kv_heads, 128, max_batch, 64, n_pages_source, n_pages_reason,
                      max_source_len, max_reason_len, max_tokens_per_call, device, pool_base, pool_bytes,
-                     rope_theta, softmax_scale, flags)
+                     rope_theta, softmax_scale, flags, position_mode, 0)
 
 
 class Context:

@@ -26,6 +26,10 @@ struct SeqState {
   std::vector<uint64_t> unit_serial;  // serial of the append call that closed unit k
   uint64_t last_src_serial = 0;       // last append call that touched this sequence
   std::vector<int32_t> pages[2];
+  // position ids of reasoning tokens in the modes other than the streaming encoding
+  int32_t concat_off = -1;            // ST_POS_CONCATENATED: T, fixed when the first reasoning token is appended
+  int32_t unit_tokens = 0;            // ST_POS_UNIT_ALIGNED: reasoning tokens of the current unit (or final stage) so far
+  int32_t final_base = -1;            // ST_POS_UNIT_ALIGNED: S, fixed at the first final-depth call
 };
 
 struct EventRec {
@@ -41,6 +45,8 @@ struct Pending {
   int next_layer = 0;
   uint32_t flags = 0;
   std::vector<int32_t> seq_ids, cu, vis_tokens;
+  std::vector<int32_t> rope_off;      // per listed sequence: position id of a new token minus its index in the cache
+  std::vector<uint8_t> is_final;      // per listed sequence: the call named ST_VIS_ALL (final depth)
   uint64_t wait_serial = 0;
 };
 
@@ -133,6 +139,8 @@ bool config_ok(const st_config *c, std::string *why) {
   if (c->max_tokens_per_call < 1) return bad("max_tokens_per_call must be >= 1");
   if (!(c->rope_theta > 0.0)) return bad("rope_theta must be > 0");
   if (c->softmax_scale < 0.f) return bad("softmax_scale must be >= 0");
+  if (c->position_mode < ST_POS_STREAMING || c->position_mode > ST_POS_UNIT_ALIGNED) return bad("unknown position_mode");
+  if (c->reserved != 0) return bad("reserved must be 0");
   return true;
 }
 
@@ -286,6 +294,31 @@ int resolve_visibility(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq, const
   return ST_OK;
 }
 
+// Position ids of the new reasoning tokens of a call (Section 3.2): offset between a token's position id and its index
+// in the reasoning cache, per listed sequence. Zero with the streaming position encoding.
+int resolve_positions(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq, const int32_t *visible_units,
+                      std::vector<int32_t> *rope_off, std::vector<uint8_t> *is_final) {
+  rope_off->assign(n_seq, 0);
+  is_final->assign(n_seq, 0);
+  for (int i = 0; i < n_seq; ++i) {
+    const SeqState &sq = ctx->seqs[seq_ids[i]];
+    (*is_final)[i] = visible_units && visible_units[i] == ST_VIS_ALL;
+    if (ctx->cfg.position_mode == ST_POS_CONCATENATED) {
+      (*rope_off)[i] = sq.concat_off >= 0 ? sq.concat_off : sq.len[0];            // T + t
+    } else if (ctx->cfg.position_mode == ST_POS_UNIT_ALIGNED) {
+      int32_t base;
+      if ((*is_final)[i]) {
+        base = sq.final_base >= 0 ? sq.final_base : sq.len[0];                      // S + i
+      } else {
+        if (sq.n_eot > sq.n_eos) return fail(ctx, ST_ERR_NOT_READY, "the source unit this reasoning unit aligns to has not been appended yet");
+        base = sq.n_eot > 0 ? sq.unit_end[sq.n_eot - 1] : 0;                        // P_{u-1} + i for unit u = N_EOT + 1
+      }
+      (*rope_off)[i] = base + sq.unit_tokens - sq.len[1];
+    }
+  }
+  return ST_OK;
+}
+
 // Make `stream` wait for the source append with the given serial if it ran on another stream.
 int wait_for_append(st_ctx *ctx, uint64_t serial, cudaStream_t stream) {
   if (int rc = injected_failure(ctx, "stream wait")) return rc;
@@ -389,7 +422,7 @@ int unstage_output(st_ctx *ctx, int side, uint32_t flags, int32_t total, void *o
 
 // Launch the append kernel (K and V into the cache of side `which`, rotated q into scratch).
 int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
-               const IoPtrs &io, bool want_q, cudaStream_t stream) {
+               const std::vector<int32_t> &rope_off, const IoPtrs &io, bool want_q, cudaStream_t stream) {
   if (int rc = injected_failure(ctx, "append launch")) return rc;
   if (ctx->host_only) return ST_OK;
   for (int s0 = 0; s0 < n_seq; s0 += st::kMaxSeqPerLaunch) {
@@ -412,7 +445,7 @@ int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, co
     for (int i = 0; i < ns; ++i) {
       const int b = s0 + i;
       const int32_t pos0 = ctx->seqs[seq_ids[b]].len[which], n = cu[b + 1] - cu[b];
-      ap.seq[i] = {seq_ids[b], pos0, n, cu[b], blocks};
+      ap.seq[i] = {seq_ids[b], pos0, n, cu[b], blocks, which == 1 ? rope_off[b] : 0};
       if (n > 0) blocks += ((pos0 + n - 1) >> 3) - (pos0 >> 3) + 1;
     }
     if (blocks == 0) continue;
@@ -451,8 +484,8 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
 // Attention for the rows of a call. kind: 0 chunk prefill, 1 decode, 2 extend.
 // `fused`: non-null for a decode step whose append runs inside the decode kernel (the call's un-rotated q/k/v).
 int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
-                  const std::vector<int32_t> &vis_tokens, float *out, uint32_t flags, cudaStream_t stream,
-                  const IoPtrs &io, bool fused) {
+                  const std::vector<int32_t> &vis_tokens, const std::vector<int32_t> &rope_off, float *out, uint32_t flags,
+                  cudaStream_t stream, const IoPtrs &io, bool fused) {
   if (int rc = injected_failure(ctx, "attention launch")) return rc;
   if (ctx->host_only || !out) return ST_OK;
   const int side = kind == 0 ? 0 : 1;
@@ -484,6 +517,7 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
       as.n_rows = n;
       as.q_begin = cu[b];
       as.work_begin = 0;
+      as.rope_off = kind == 0 ? 0 : rope_off[b];
       ap.seq[n_used++] = as;
     }
     if (n_used == 0) continue;
@@ -515,7 +549,7 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
 }
 
 void record_meta(st_ctx *ctx, int kind, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
-                 const std::vector<int32_t> &vis_tokens) {
+                 const std::vector<int32_t> &vis_tokens, const std::vector<int32_t> &rope_off) {
   const int side = kind == 0 ? 0 : 1;
   const int total = cu[n_seq];
   ctx->meta_pos.assign(total, 0);
@@ -525,7 +559,7 @@ void record_meta(st_ctx *ctx, int kind, const int32_t *seq_ids, const int32_t *c
     const int32_t base = ctx->seqs[seq_ids[b]].len[side];
     for (int r = cu[b]; r < cu[b + 1]; ++r) {
       const int32_t pos = base + (r - cu[b]);
-      ctx->meta_pos[r] = pos;
+      ctx->meta_pos[r] = pos + (kind == 0 ? 0 : rope_off[b]);
       if (kind == 0) {
         ctx->meta_vis_src[r] = pos + 1;
         ctx->meta_vis_rsn[r] = 0;
@@ -556,8 +590,11 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
   if (layer == 0) {
     std::vector<int32_t> vis;
     uint64_t wait_serial = 0;
+    std::vector<int32_t> off(n_seq, 0);
+    std::vector<uint8_t> fin(n_seq, 0);
     if (kind != 0) {
       if ((rc = resolve_visibility(ctx, seq_ids, n_seq, visible_units, &vis, &wait_serial))) return rc;
+      if ((rc = resolve_positions(ctx, seq_ids, n_seq, visible_units, &off, &fin))) return rc;
     }
     if ((rc = plan_pages(ctx, side, seq_ids, cu, n_seq, &updates))) return rc;
     pd.active = true;
@@ -567,8 +604,10 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     pd.seq_ids.assign(seq_ids, seq_ids + n_seq);
     pd.cu.assign(cu, cu + n_seq + 1);
     pd.vis_tokens = vis;
+    pd.rope_off = off;
+    pd.is_final = fin;
     pd.wait_serial = wait_serial;
-    record_meta(ctx, kind, seq_ids, cu, n_seq, pd.vis_tokens);
+    record_meta(ctx, kind, seq_ids, cu, n_seq, pd.vis_tokens, pd.rope_off);
   }
 
   // Device steps. If one of them fails, the host-side plan of this call is taken back (pages to the free list, the
@@ -588,8 +627,8 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     // decode step whose append is not fused, and the tensor-core kernel's two-term variant (which wants the fp64
     // rotation). The one-term tensor-core kernel rotates its own.
     const bool want_qhat = io.out != nullptr && ((flags & ST_REFERENCE_KERNELS) || kind == 1 || ctx->precise_p);
-    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, io, want_qhat, stream))) return r;
-    if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, io.out, flags, stream, io, fuse_append))) return r;
+    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, pd.rope_off, io, want_qhat, stream))) return r;
+    if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, pd.rope_off, io.out, flags, stream, io, fuse_append))) return r;
     if ((r = unstage_output(ctx, side, flags, total, out, stream, io))) return r;
     if (layer == ctx->cfg.n_layers - 1 && kind == 0 && !ctx->host_only) {
       // the event later reasoning-side calls on another stream wait for
@@ -627,8 +666,15 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
           sq.unit_end.push_back(sq.len[0]);
           sq.unit_serial.push_back(serial);
         }
-      } else if (flags & ST_END_OF_UNIT) {
-        ++sq.n_eot;
+      } else {
+        // position-id bookkeeping of the other modes (the streaming encoding needs none)
+        if (ctx->cfg.position_mode == ST_POS_CONCATENATED && sq.concat_off < 0 && cu[b + 1] > cu[b]) sq.concat_off = pd.rope_off[b];
+        if (pd.is_final[b] && sq.final_base < 0) sq.final_base = sq.len[0];
+        sq.unit_tokens += cu[b + 1] - cu[b];
+        if (flags & ST_END_OF_UNIT) {
+          ++sq.n_eot;
+          sq.unit_tokens = 0;
+        }
       }
     }
     pd.active = false;
@@ -742,7 +788,8 @@ int st_create(const st_config *cfg, st_ctx **out) {
     ST_CREATE_CUDA(cudaMalloc(&ctx->partial, sizeof(float) * st::decode_partial_floats(st::kMaxSeqPerLaunch, cfg->n_kv_heads, ctx->num_sms)));
     {
       // a reasoning position is below the page table's reach: ptab_stride pages of 64 tokens
-      const int n_hi = (int)(((int64_t)ctx->ptab_stride[1] * 64 + st::kRopeLoSteps - 1) / st::kRopeLoSteps) + 1;
+      // (with the concatenated or unit-aligned position ids a reasoning token's position may also count source tokens)
+      const int n_hi = (int)(((int64_t)(ctx->ptab_stride[0] + ctx->ptab_stride[1]) * 64 + st::kRopeLoSteps - 1) / st::kRopeLoSteps) + 1;
       ST_CREATE_CUDA(cudaMalloc(&ctx->rope_hi, sizeof(double2) * 64 * (size_t)n_hi));
       ST_CREATE_CUDA(cudaMalloc(&ctx->rope_lo, sizeof(double2) * 64 * (size_t)st::kRopeLoSteps));
       ST_CREATE_CUDA(st::launch_rope_table(ctx->inv_freq, ctx->rope_hi, n_hi, st::kRopeLoSteps, nullptr));

@@ -381,7 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         for (int it = r_local; it < n_items; it += kRowsPerTile) {
           const int tk = tok_lo + (it >> 3), c = it & 7;
           float cs[8], sn[8];
-          const double pos = (double)(sq.b_base + tk);
+          const double pos = (double)(sq.b_base + tk + sq.rope_off);
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const double turns = pos * p.inv_freq[8 * c + e] * 0.15915494309189535;   // angle / 2 pi

@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256) st_k_rope_append(const __grid_constant__ 
   for (int i = threadIdx.x; i < nt * 64; i += blockDim.x) {
     const int t = i >> 6, c = i & 63;
     double sn, cs;
-    sincos((double)(pos_lo + t) * p.inv_freq[c], &sn, &cs);
+    sincos((double)(pos_lo + t + sq.rope_off) * p.inv_freq[c], &sn, &cs);
     s_cos[t][c] = cs;
     s_sin[t][c] = sn;
   }

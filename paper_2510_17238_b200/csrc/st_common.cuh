@@ -57,6 +57,7 @@ struct AppendSeq {
   int32_t n;          // new tokens of this sequence
   int32_t q_begin;    // first packed row of this sequence in q/k/v
   int32_t blk_begin;  // first thread block of this sequence (blocks cover aligned groups of 8 positions)
+  int32_t rope_off;   // position id of a token = its index in the cache + rope_off (0 with the streaming position encoding)
 };
 
 struct AppendParams {
@@ -83,6 +84,7 @@ struct AttnSeq {
   int32_t n_rows;
   int32_t q_begin;    // first packed row in qhat / out
   int32_t work_begin; // kernel specific prefix (tiles or blocks)
+  int32_t rope_off;   // position id of row i = b_base + i + rope_off (kernels that rotate their own queries or keys)
 };
 
 struct AttnParams {

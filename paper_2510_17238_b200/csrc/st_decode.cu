@@ -208,15 +208,16 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
           if (lane == 0) good = mbar_wait(smem_u32(&sm.q_free[slot]), (uint32_t)(use - 1) & 1u, abort_flag, p.status, kDevTimeoutDecode);
           if (!__shfl_sync(0xffffffffu, good, 0)) break;
         }
-        const int pos = sq.b_base;                  // position of the step's token in the reasoning stream
+        const int pos = sq.b_base;                  // index of the step's token in the reasoning cache
+        const int rpos = pos + sq.rope_off;         // its position id
         // every global load of the pair is issued before the first value is used: one round trip, not five
         double2 hi[2], lo[2];
         __nv_bfloat16 qx[8][2], qy[8][2], kx[2], ky[2], vv[4];
         int page = 0;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          hi[i] = p.rope_hi[(size_t)(pos / kRopeLoSteps) * 64 + lane + 32 * i];
-          lo[i] = p.rope_lo[(size_t)(pos % kRopeLoSteps) * 64 + lane + 32 * i];
+          hi[i] = p.rope_hi[(size_t)(rpos / kRopeLoSteps) * 64 + lane + 32 * i];
+          lo[i] = p.rope_lo[(size_t)(rpos % kRopeLoSteps) * 64 + lane + 32 * i];
         }
 #pragma unroll
         for (int g = 0; g < 8; ++g) {

@@ -145,6 +145,7 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
     p.seq[i].n_rows = 1;
     p.seq[i].q_begin = i;
     p.seq[i].work_begin = 0;
+    p.seq[i].rope_off = 0;
   }
   cudaStream_t s = (cudaStream_t)stream;
   // the status word is the only part of the workspace that must start at zero; partial records are

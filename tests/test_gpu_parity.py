@@ -129,6 +129,23 @@ def test_eq2_literal_lag_and_input_far_ahead():
     pu.check_against_oracle(w1, s1, plan, batches[0], flats[0], n_random=64, full_seqs=(1,), what="cfg1 lookahead 3")
 
 
+@pytest.mark.parametrize("position_mode", [api.ST_POS_CONCATENATED, api.ST_POS_UNIT_ALIGNED])
+def test_other_position_modes(position_mode):
+    """The original RoPE ids (reasoning token t at T + t, whole input appended first: the batch setting in which the
+    paper compares the encodings) and the unit-aligned variant: rows and both caches against the oracle with the same
+    ids, token by token (the decode kernel's fused append) and span by span (append kernel + tensor-core kernel)."""
+    w = small_workload(32)
+    scheds = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0),
+              workloads.SeqSchedule((200, 56), (70, 9), 66)]
+    lookahead = 4 if position_mode == api.ST_POS_CONCATENATED else 2
+    for mode in ("decode", "extend"):
+        ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode=mode, lookahead=lookahead, position_mode=position_mode)
+        pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], what=f"position mode {position_mode} {mode}",
+                                position_mode=position_mode)
+        assert pu.check_cache(ctx, w, scheds, plan, flats[0], position_mode=position_mode) <= 2
+        ctx.close()
+
+
 def test_page_id_outside_the_pool_is_reported_not_dereferenced():
     """The kernels compare every page id they read with the pool's page count before they build an address from it.
     The test overwrites one entry of the device page table with an id far outside the pool (a host-side test hook,

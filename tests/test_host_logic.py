@@ -117,13 +117,18 @@ def test_workload_recipes():
     assert (q == q2).all()
 
 
-def drive_plan_host_only(scheds, mode, n_layers=1, lookahead=1):
+POSITION_MODE_NAMES = {api.ST_POS_STREAMING: "streaming", api.ST_POS_CONCATENATED: "concatenated",
+                       api.ST_POS_UNIT_ALIGNED: "unit_aligned"}
+
+
+def drive_plan_host_only(scheds, mode, n_layers=1, lookahead=1, position_mode=api.ST_POS_STREAMING):
     """Replays a plan on a host-only context and checks, call by call, that the positions and
     visibility the kernels would receive equal the oracle's schedule."""
     plan = runner.make_plan(scheds, mode=mode, lookahead=lookahead)
     w = workloads.WORKLOADS[0]
-    ctx = runner.make_context(w, scheds, plan, n_layers=n_layers, flags=api.ST_CFG_HOST_ONLY)
-    oracles = [osa.build_schedule(s.src_unit_len, s.rsn_unit_len, s.final_len) for s in scheds]
+    ctx = runner.make_context(w, scheds, plan, n_layers=n_layers, flags=api.ST_CFG_HOST_ONLY, position_mode=position_mode)
+    oracles = [osa.build_schedule(s.src_unit_len, s.rsn_unit_len, s.final_len,
+                                  position_mode=POSITION_MODE_NAMES[position_mode]) for s in scheds]
     src_i = rsn_i = 0
     for call in plan.calls:
         for layer in range(n_layers):
@@ -172,6 +177,20 @@ def test_plan_positions_and_visibility_bit_exact_ragged(mode):
               for b, s in enumerate(full)]
     scheds[1] = workloads.SeqSchedule(scheds[1].src_unit_len, (0, 3, 0, 2), 0)
     drive_plan_host_only(scheds, mode)
+
+
+@pytest.mark.parametrize("mode", ["decode", "extend"])
+def test_plan_positions_in_the_other_position_modes(mode):
+    """Original RoPE ids (reasoning token t at T + t; the whole input is appended first, as in the batch setting the
+    paper compares the encodings in) and the unit-aligned variant, call by call against the oracle's ids."""
+    uniform = [workloads.scaled_schedule(3, 70, 5, 9)] * 2
+    ragged = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0)]
+    drive_plan_host_only(uniform, mode, lookahead=3, position_mode=api.ST_POS_CONCATENATED)
+    drive_plan_host_only(ragged, mode, n_layers=2, lookahead=4, position_mode=api.ST_POS_CONCATENATED)
+    drive_plan_host_only(uniform, mode, n_layers=2, position_mode=api.ST_POS_UNIT_ALIGNED)
+    drive_plan_host_only(ragged, mode, lookahead=2, position_mode=api.ST_POS_UNIT_ALIGNED)
+    with pytest.raises(api.StError):
+        host_ctx(position_mode=7)
 
 
 def test_algorithm1_counters_and_not_ready():
