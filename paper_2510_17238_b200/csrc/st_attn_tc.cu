@@ -310,6 +310,29 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
   }
   const int n_max = (n_pages + 1) >> 1;
 
+  // Q rows of M-tile t into the swizzled operand layout, by asynchronous 16-byte copies: the tile's 128 threads copy it
+  // 8 rows at a time, 16 lanes take the 16 chunks of one row, so every copy instruction reads whole 256-byte rows; rows
+  // past the end of the sequence are zero-filled (source size 0, nothing is read).
+  auto issue_q_copies = [&](int t, int r_local) {
+    const __nv_bfloat16 *q_src = kPrecise ? p.qhat : p.q_raw;
+    const int c = r_local & 15;                            // chunk of the row
+    const uint32_t q_smem = smem_u32(smem + kOffQ + t * kQTileBytes);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int rr = i * 8 + (r_local >> 4);                // row of the tile
+      const int grow = row0 + t * kRowsPerTile + rr;
+      const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
+      const bool in = grow < packed_rows;
+      const __nv_bfloat16 *src = in ? q_src + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + c * 8 : q_src;
+      cp_async16(q_smem + (c >> 3) * kHalfPanel + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src, in ? 16u : 0u);
+    }
+  };
+  // The one-term variant reads the caller's un-rotated queries, which no kernel in front of this one writes: their
+  // copies start at once and fly while the barriers and the tensor memory are set up (about 2,000 cycles).
+  if constexpr (!kPrecise) {
+    if (warp < 8 && active[warp >> 2]) issue_q_copies(warp >> 2, (warp & 3) * 32 + lane);
+  }
+
   // one thread per barrier (24 of them: a single thread took ~600 cycles over this). Barriers that the four softmax
   // warps of an M-tile arrive at count 4, those completed by tcgen05.commit or a bulk copy count 1.
   constexpr int kNumBarriers = (int)(offsetof(Barriers, tmem_base) / sizeof(uint64_t));
@@ -351,18 +374,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       // One-term variant: the rows come un-rotated from the caller's buffer and are rotated in place below.
       uint8_t *q_tile = smem + kOffQ + t * kQTileBytes;
       {
-        const __nv_bfloat16 *q_src = kPrecise ? p.qhat : p.q_raw;
-        const int c = r_local & 15;                          // chunk of the row
-        const uint32_t q_smem = smem_u32(q_tile);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int rr = i * 8 + (r_local >> 4);              // row of the tile
-          const int grow = row0 + t * kRowsPerTile + rr;
-          const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
-          const bool in = grow < packed_rows;
-          const __nv_bfloat16 *src = in ? q_src + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + c * 8 : q_src;
-          cp_async16(q_smem + (c >> 3) * kHalfPanel + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src, in ? 16u : 0u);
-        }
+        if constexpr (kPrecise) issue_q_copies(t, r_local);   // (the one-term variant issued them before the set-up)
         cp_async_wait_all();
       }
       if constexpr (!kPrecise) {
