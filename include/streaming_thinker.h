@@ -179,6 +179,24 @@ ST_API int st_reason_extend(st_ctx *ctx, int32_t layer,
                      const void *q, const void *k, const void *v, void *out,
                      uint32_t flags, void *stream);
 
+/* One pass over the training layout of Section 3.2 (the layout Eq. 2's mask is written on): for every listed
+ * sequence the packed rows are [all source tokens ; all reasoning tokens], sequence after sequence in q/k/v/out
+ * (device, as in the other calls; the total row count is bounded by max_tokens_per_call). The schedule comes as in
+ * st_schedule_build, for n_seq sequences: n_units[b] units per sequence, their source and reasoning lengths
+ * concatenated over the sequences in src_unit_len / rsn_unit_len (host arrays of sum(n_units) ints), final_len[b]
+ * final-depth tokens, lag_units as in st_schedule_build. Every source row attends causally to the source tokens
+ * (Eq. 2's unmodified part); every reasoning row of unit u attends to the source prefix of unit min(u + lag, U)
+ * (Eq. 1 / the streaming mask region) and causally to the reasoning tokens; final-depth rows see the whole source.
+ * Position ids follow the context's position_mode (streaming or concatenated; the unit-aligned variant is not
+ * supported here). Forward only. The listed sequences must be empty; afterwards both caches hold the whole
+ * sequence with N_EOS = N_EOT = n_units[b], exactly as if the units had been streamed in, so decoding can go on from
+ * there. Multi-layer contexts: one call per layer, in order, with identical arguments. flags: ST_REFERENCE_KERNELS,
+ * ST_IO_HOST. out may be NULL (caches only). */
+ST_API int st_forward_packed(st_ctx *ctx, int32_t layer, const int32_t *seq_ids, int32_t n_seq, const int32_t *n_units,
+                             const int32_t *src_unit_len, const int32_t *rsn_unit_len, const int32_t *final_len,
+                             int32_t lag_units, const void *q, const void *k, const void *v, void *out, uint32_t flags,
+                             void *stream);
+
 /* Schedule generator (pure host, no context): turns a streaming-unit schedule -- n_units source-unit
  * lengths, the reasoning-unit length that follows each, and final_len final-depth tokens -- into the
  * paper's position ids and visibility. With S = sum(src_unit_len), R = sum(rsn_unit_len) + final_len:

@@ -54,6 +54,8 @@ _SIGS = {
     "st_append_source_chunk": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, _vp, _vp, _vp, _vp, C.c_uint32, _vp]),
     "st_reason_decode": (C.c_int, [_vp, C.c_int32, _i32p, C.c_int32, _i32p, _vp, _vp, _vp, _vp, C.c_uint32, _vp]),
     "st_reason_extend": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, _i32p, _vp, _vp, _vp, _vp, C.c_uint32, _vp]),
+    "st_forward_packed": (C.c_int, [_vp, C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, C.c_int32, _vp, _vp, _vp, _vp,
+                                    C.c_uint32, _vp]),
     "st_schedule_build": (C.c_int, [_i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, _i32p, _i32p, _i64p, _i64p]),
     "st_schedule_dense_mask": (C.c_int, [_i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_uint8)]),
     "st_seq_state": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, _i32p, _i32p]),
@@ -170,6 +172,17 @@ class Context:
         pv, kv = _i32(visible_units)
         rc = lib.st_reason_extend(self._h, layer, ps, pc, len(ks), pv, _ptr(q), _ptr(k), _ptr(v), _ptr(out), flags,
                                   _ptr(stream))
+        return self._check(rc) if check else rc
+
+    def forward_packed(self, layer, seq_ids, scheds, q, k, v, out, lag_units=0, flags=0, stream=None, check=True):
+        """st_forward_packed for a list of schedules (objects with src_unit_len, rsn_unit_len, final_len)."""
+        ps, ks = _i32(seq_ids)
+        pn, kn = _i32([len(s.src_unit_len) for s in scheds])
+        pa, ka = _i32([x for s in scheds for x in s.src_unit_len] or [0])
+        pb, kb = _i32([x for s in scheds for x in s.rsn_unit_len] or [0])
+        pf, kf = _i32([s.final_len for s in scheds])
+        rc = lib.st_forward_packed(self._h, layer, ps, len(ks), pn, pa, pb, pf, lag_units, _ptr(q), _ptr(k), _ptr(v),
+                                   _ptr(out), flags, _ptr(stream))
         return self._check(rc) if check else rc
 
     def seq_state(self, seq_id):

@@ -351,6 +351,22 @@ int wait_for_append(st_ctx *ctx, uint64_t serial, cudaStream_t stream) {
   return ST_OK;
 }
 
+// After the last layer of a source append: the event that later reasoning-side calls on another stream wait for.
+int record_append_event(st_ctx *ctx, cudaStream_t stream) {
+  if (ctx->host_only) return ST_OK;
+  EventRec &rec = ctx->events[(ctx->serial + 1) % kEventRing];
+  if (ctx->cross_stream) {
+    if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
+    ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
+    rec.stream = stream;
+    rec.serial = ctx->serial + 1;
+  } else {
+    rec.serial = 0;   // none recorded: wait_for_append falls back to the catch-all event
+  }
+  ctx->last_src_stream = stream;
+  return ST_OK;
+}
+
 struct IoPtrs {
   const __nv_bfloat16 *q, *k, *v;
   float *out;
@@ -421,7 +437,19 @@ int unstage_output(st_ctx *ctx, int side, uint32_t flags, int32_t total, void *o
 }
 
 // Launch the append kernel (K and V into the cache of side `which`, rotated q into scratch).
-int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
+// Rows of a call per listed sequence: first packed row and row count.
+struct RowRanges {
+  std::vector<int32_t> begin, count;
+  static RowRanges from_cu(const int32_t *cu, int32_t n_seq) {
+    RowRanges r;
+    r.begin.assign(cu, cu + n_seq);
+    r.count.resize(n_seq);
+    for (int b = 0; b < n_seq; ++b) r.count[b] = cu[b + 1] - cu[b];
+    return r;
+  }
+};
+
+int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, const RowRanges &rows, int32_t n_seq,
                const std::vector<int32_t> &rope_off, const IoPtrs &io, bool want_q, cudaStream_t stream) {
   if (int rc = injected_failure(ctx, "append launch")) return rc;
   if (ctx->host_only) return ST_OK;
@@ -444,8 +472,8 @@ int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, co
     int blocks = 0;
     for (int i = 0; i < ns; ++i) {
       const int b = s0 + i;
-      const int32_t pos0 = ctx->seqs[seq_ids[b]].len[which], n = cu[b + 1] - cu[b];
-      ap.seq[i] = {seq_ids[b], pos0, n, cu[b], blocks, which == 1 ? rope_off[b] : 0};
+      const int32_t pos0 = ctx->seqs[seq_ids[b]].len[which], n = rows.count[b];
+      ap.seq[i] = {seq_ids[b], pos0, n, rows.begin[b], blocks, which == 1 ? rope_off[b] : 0};
       if (n > 0) blocks += ((pos0 + n - 1) >> 3) - (pos0 >> 3) + 1;
     }
     if (blocks == 0) continue;
@@ -483,16 +511,14 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
 
 // Attention for the rows of a call. kind: 0 chunk prefill, 1 decode, 2 extend.
 // `fused`: non-null for a decode step whose append runs inside the decode kernel (the call's un-rotated q/k/v).
-int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
-                  const std::vector<int32_t> &vis_tokens, const std::vector<int32_t> &rope_off, float *out, uint32_t flags,
-                  cudaStream_t stream, const IoPtrs &io, bool fused) {
-  if (int rc = injected_failure(ctx, "attention launch")) return rc;
-  if (ctx->host_only || !out) return ST_OK;
+// Launches the attention kernels of one call for a list of work entries (one per sequence for the streaming calls,
+// one per (sequence, reasoning unit) for the packed forward). kind: 0 chunk prefill, 1 decode, 2 spans.
+// `fused`: a decode step whose append runs inside the decode kernel (the call's un-rotated q/k/v).
+int launch_attention_entries(st_ctx *ctx, int kind, int32_t layer, const std::vector<st::AttnSeq> &entries, int total_rows,
+                             float *out, uint32_t flags, cudaStream_t stream, const IoPtrs &io, bool fused) {
   const int side = kind == 0 ? 0 : 1;
-  const int total_rows = cu[n_seq];
-  if (total_rows == 0) return ST_OK;
-  for (int s0 = 0; s0 < n_seq; s0 += st::kMaxSeqPerLaunch) {
-    const int ns = std::min<int>(st::kMaxSeqPerLaunch, n_seq - s0);
+  for (size_t s0 = 0; s0 < entries.size(); s0 += st::kMaxSeqPerLaunch) {
+    const int ns = (int)std::min<size_t>(st::kMaxSeqPerLaunch, entries.size() - s0);
     st::AttnParams ap;
     fill_attn_common(ctx, side, layer, out, &ap);
     if (fused) {
@@ -504,24 +530,8 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
     } else if (kind != 1 && !(flags & ST_REFERENCE_KERNELS)) {
       ap.q_raw = io.q;   // the tensor-core kernel rotates its query rows itself
     }
-    int n_used = 0;
-    for (int i = 0; i < ns; ++i) {
-      const int b = s0 + i;
-      const int32_t n = cu[b + 1] - cu[b];
-      if (n == 0) continue;
-      const SeqState &sq = ctx->seqs[seq_ids[b]];
-      st::AttnSeq as;
-      as.slot = seq_ids[b];
-      as.a_len = kind == 0 ? 0 : vis_tokens[b];
-      as.b_base = sq.len[side];
-      as.n_rows = n;
-      as.q_begin = cu[b];
-      as.work_begin = 0;
-      as.rope_off = kind == 0 ? 0 : rope_off[b];
-      ap.seq[n_used++] = as;
-    }
-    if (n_used == 0) continue;
-    ap.n_seq = n_used;
+    std::copy(entries.begin() + s0, entries.begin() + s0 + ns, ap.seq);
+    ap.n_seq = ns;
     int nl = 0;
     cudaEvent_t t0 = nullptr, t1 = nullptr;
     if (ctx->timing && !(flags & ST_REFERENCE_KERNELS) && (kind != 1 || ctx->timing_seen++ % ctx->timing == 0)) {
@@ -546,6 +556,31 @@ int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, 
     ctx->launches += nl;
   }
   return ST_OK;
+}
+
+// Attention for the rows of a streaming call: one entry per listed sequence with rows.
+int run_attention(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
+                  const std::vector<int32_t> &vis_tokens, const std::vector<int32_t> &rope_off, float *out, uint32_t flags,
+                  cudaStream_t stream, const IoPtrs &io, bool fused) {
+  if (int rc = injected_failure(ctx, "attention launch")) return rc;
+  if (ctx->host_only || !out) return ST_OK;
+  const int side = kind == 0 ? 0 : 1;
+  if (cu[n_seq] == 0) return ST_OK;
+  std::vector<st::AttnSeq> entries;
+  for (int b = 0; b < n_seq; ++b) {
+    const int32_t n = cu[b + 1] - cu[b];
+    if (n == 0) continue;
+    st::AttnSeq as;
+    as.slot = seq_ids[b];
+    as.a_len = kind == 0 ? 0 : vis_tokens[b];
+    as.b_base = ctx->seqs[seq_ids[b]].len[side];
+    as.n_rows = n;
+    as.q_begin = cu[b];
+    as.work_begin = 0;
+    as.rope_off = kind == 0 ? 0 : rope_off[b];
+    entries.push_back(as);
+  }
+  return launch_attention_entries(ctx, kind, layer, entries, cu[n_seq], out, flags, stream, io, fused);
 }
 
 void record_meta(st_ctx *ctx, int kind, const int32_t *seq_ids, const int32_t *cu, int32_t n_seq,
@@ -627,22 +662,10 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     // decode step whose append is not fused, and the tensor-core kernel's two-term variant (which wants the fp64
     // rotation). The one-term tensor-core kernel rotates its own.
     const bool want_qhat = io.out != nullptr && ((flags & ST_REFERENCE_KERNELS) || kind == 1 || ctx->precise_p);
-    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, cu, n_seq, pd.rope_off, io, want_qhat, stream))) return r;
+    if (!fuse_append && (r = run_append(ctx, side, layer, seq_ids, RowRanges::from_cu(cu, n_seq), n_seq, pd.rope_off, io, want_qhat, stream))) return r;
     if ((r = run_attention(ctx, kind, layer, seq_ids, cu, n_seq, pd.vis_tokens, pd.rope_off, io.out, flags, stream, io, fuse_append))) return r;
     if ((r = unstage_output(ctx, side, flags, total, out, stream, io))) return r;
-    if (layer == ctx->cfg.n_layers - 1 && kind == 0 && !ctx->host_only) {
-      // the event later reasoning-side calls on another stream wait for
-      EventRec &rec = ctx->events[(ctx->serial + 1) % kEventRing];
-      if (ctx->cross_stream) {
-        if (!rec.ev) ST_CUDA(ctx, cudaEventCreateWithFlags(&rec.ev, cudaEventDisableTiming));
-        ST_CUDA(ctx, cudaEventRecord(rec.ev, stream));
-        rec.stream = stream;
-        rec.serial = ctx->serial + 1;
-      } else {
-        rec.serial = 0;   // none recorded: wait_for_append falls back to the catch-all event
-      }
-      ctx->last_src_stream = stream;
-    }
+    if (layer == ctx->cfg.n_layers - 1 && kind == 0 && (r = record_append_event(ctx, stream))) return r;
     return ST_OK;
   };
   if ((rc = device_steps())) {
@@ -678,6 +701,160 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
       }
     }
     pd.active = false;
+  } else {
+    pd.next_layer = layer + 1;
+  }
+  return ST_OK;
+}
+
+// st_forward_packed: one pass over the training layout [source ; reasoning] of every listed sequence.
+int forward_packed(st_ctx *ctx, int32_t layer, const int32_t *seq_ids, int32_t n_seq, const int32_t *n_units,
+                   const int32_t *src_unit_len, const int32_t *rsn_unit_len, const int32_t *final_len, int32_t lag_units,
+                   const void *q, const void *k, const void *v, void *out, uint32_t flags, cudaStream_t stream) {
+  int rc = check_common(ctx, layer, seq_ids, n_seq);
+  if (rc) return rc;
+  if (flags & ~(ST_REFERENCE_KERNELS | ST_IO_HOST)) return fail(ctx, ST_ERR_INVALID_ARG, "unknown flag");
+  if (!n_units || !final_len || lag_units < 0) return fail(ctx, ST_ERR_INVALID_ARG, "n_units and final_len must be non-NULL, lag_units >= 0");
+  if (ctx->cfg.position_mode == ST_POS_UNIT_ALIGNED)
+    return fail(ctx, ST_ERR_INVALID_ARG, "the packed forward supports the streaming and the concatenated position ids");
+  // per sequence: S, R, first row in the packed tensors; the schedule signature for the layer protocol
+  std::vector<int32_t> S(n_seq), R(n_seq), row0(n_seq), unit0(n_seq), cu_src(n_seq + 1, 0), cu_rsn(n_seq + 1, 0), sig;
+  int64_t total = 0, units = 0;
+  for (int b = 0; b < n_seq; ++b) {
+    if (n_units[b] < 0 || final_len[b] < 0) return fail(ctx, ST_ERR_INVALID_ARG, "unit counts and final lengths must be >= 0");
+    if (n_units[b] > 0 && (!src_unit_len || !rsn_unit_len)) return fail(ctx, ST_ERR_INVALID_ARG, "unit length arrays are NULL");
+    unit0[b] = (int32_t)units;
+    int64_t s_len = 0, r_len = final_len[b];
+    for (int u = 0; u < n_units[b]; ++u) {
+      const int32_t n = src_unit_len[units + u], m = rsn_unit_len[units + u];
+      if (n < 0 || m < 0) return fail(ctx, ST_ERR_INVALID_ARG, "unit lengths must be >= 0");
+      s_len += n;
+      r_len += m;
+      sig.push_back(n);
+      sig.push_back(m);
+    }
+    sig.push_back(final_len[b]);
+    units += n_units[b];
+    if (total + s_len + r_len > ctx->cfg.max_tokens_per_call) return fail(ctx, ST_ERR_INVALID_ARG, "more tokens than max_tokens_per_call");
+    S[b] = (int32_t)s_len;
+    R[b] = (int32_t)r_len;
+    row0[b] = (int32_t)total;
+    total += s_len + r_len;
+    cu_src[b + 1] = cu_src[b] + S[b];
+    cu_rsn[b + 1] = cu_rsn[b] + R[b];
+  }
+  sig.push_back(lag_units);
+  if (total > 0 && (!q || !k || !v) && !ctx->host_only) return fail(ctx, ST_ERR_INVALID_ARG, "q, k and v must be non-NULL");
+
+  // layer protocol: the step occupies both sides
+  Pending &pd = ctx->pend[0];
+  if (layer == 0) {
+    if (pd.active || ctx->pend[1].active) return fail(ctx, ST_ERR_STATE, "previous step has not been issued for all layers");
+    for (int b = 0; b < n_seq; ++b) {
+      const SeqState &sq = ctx->seqs[seq_ids[b]];
+      if (sq.len[0] || sq.len[1] || sq.n_eos || sq.n_eot) return fail(ctx, ST_ERR_STATE, "the packed forward needs empty sequences (st_reset them first)");
+    }
+  } else {
+    if (!pd.active || pd.kind != 3 || pd.next_layer != layer) return fail(ctx, ST_ERR_STATE, "layer issued out of order");
+    if ((int)pd.seq_ids.size() != n_seq || !std::equal(pd.seq_ids.begin(), pd.seq_ids.end(), seq_ids) || pd.cu != sig)
+      return fail(ctx, ST_ERR_STATE, "step arguments differ from those given for layer 0");
+  }
+  std::vector<st::PageUpdate> updates;
+  if (layer == 0) {
+    if ((rc = plan_pages(ctx, 0, seq_ids, cu_src.data(), n_seq, &updates))) return rc;
+    if ((rc = plan_pages(ctx, 1, seq_ids, cu_rsn.data(), n_seq, &updates))) {
+      unplan_pages(ctx, updates);
+      return rc;
+    }
+    pd.active = ctx->pend[1].active = true;
+    pd.kind = 3;
+    pd.next_layer = 0;
+    pd.flags = flags;
+    pd.seq_ids.assign(seq_ids, seq_ids + n_seq);
+    pd.cu = sig;
+  }
+
+  // work entries of the reasoning rows: one per (sequence, reasoning unit with tokens), one for the final-depth tokens
+  const bool concat = ctx->cfg.position_mode == ST_POS_CONCATENATED;
+  std::vector<st::AttnSeq> src_entries, rsn_entries;
+  std::vector<int32_t> rsn_off(n_seq, 0);
+  ctx->meta_pos.assign((size_t)total, 0);
+  ctx->meta_vis_src.assign((size_t)total, 0);
+  ctx->meta_vis_rsn.assign((size_t)total, 0);
+  for (int b = 0; b < n_seq; ++b) {
+    rsn_off[b] = concat ? S[b] : 0;
+    if (S[b] > 0) src_entries.push_back({seq_ids[b], 0, 0, S[b], row0[b], 0, 0});
+    for (int j = 0; j < S[b]; ++j) {
+      ctx->meta_pos[row0[b] + j] = j;
+      ctx->meta_vis_src[row0[b] + j] = j + 1;
+    }
+    std::vector<int32_t> prefix(n_units[b] + 1, 0);
+    for (int u = 0; u < n_units[b]; ++u) prefix[u + 1] = prefix[u] + src_unit_len[unit0[b] + u];
+    int32_t r = 0;
+    for (int u = 0; u <= n_units[b]; ++u) {
+      const bool fin = u == n_units[b];
+      const int32_t m = fin ? final_len[b] : rsn_unit_len[unit0[b] + u];
+      const int32_t vis = fin ? S[b] : prefix[std::min<int64_t>((int64_t)u + 1 + lag_units, n_units[b])];
+      if (m > 0) rsn_entries.push_back({seq_ids[b], vis, r, m, row0[b] + S[b] + r, 0, rsn_off[b]});
+      for (int i = 0; i < m; ++i) {
+        const int32_t row = row0[b] + S[b] + r + i;
+        ctx->meta_pos[row] = r + i + rsn_off[b];
+        ctx->meta_vis_src[row] = vis;
+        ctx->meta_vis_rsn[row] = r + i + 1;
+      }
+      r += m;
+    }
+  }
+
+  auto device_steps = [&]() -> int {
+    int r;
+    if (!ctx->host_only) ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if ((r = push_page_updates(ctx, updates, stream))) return r;
+    IoPtrs io;
+    if ((r = stage_inputs(ctx, 0, flags, (int32_t)total, q, k, v, out, stream, &io))) return r;
+    const bool want_qhat = io.out != nullptr && ((flags & ST_REFERENCE_KERNELS) || ctx->precise_p);
+    RowRanges src_rows, rsn_rows;
+    for (int b = 0; b < n_seq; ++b) {
+      src_rows.begin.push_back(row0[b]);
+      src_rows.count.push_back(S[b]);
+      rsn_rows.begin.push_back(row0[b] + S[b]);
+      rsn_rows.count.push_back(R[b]);
+    }
+    if ((r = run_append(ctx, 0, layer, seq_ids, src_rows, n_seq, rsn_off, io, want_qhat, stream))) return r;
+    if ((r = run_append(ctx, 1, layer, seq_ids, rsn_rows, n_seq, rsn_off, io, want_qhat, stream))) return r;
+    if ((r = injected_failure(ctx, "attention launch"))) return r;
+    if (!ctx->host_only && io.out) {
+      if ((r = launch_attention_entries(ctx, 0, layer, src_entries, (int)total, io.out, flags, stream, io, false))) return r;
+      if ((r = launch_attention_entries(ctx, 2, layer, rsn_entries, (int)total, io.out, flags, stream, io, false))) return r;
+    }
+    if ((r = unstage_output(ctx, 0, flags, (int32_t)total, out, stream, io))) return r;
+    if (layer == ctx->cfg.n_layers - 1 && (r = record_append_event(ctx, stream))) return r;
+    return ST_OK;
+  };
+  if ((rc = device_steps())) {
+    if (layer == 0) {
+      unplan_pages(ctx, updates);
+      pd.active = ctx->pend[1].active = false;
+    }
+    return rc;
+  }
+  if (layer == ctx->cfg.n_layers - 1) {
+    const uint64_t serial = ++ctx->serial;
+    for (int b = 0; b < n_seq; ++b) {
+      SeqState &sq = ctx->seqs[seq_ids[b]];
+      sq.len[0] = S[b];
+      sq.len[1] = R[b];
+      sq.last_src_serial = serial;
+      int32_t p = 0;
+      for (int u = 0; u < n_units[b]; ++u) {
+        p += src_unit_len[unit0[b] + u];
+        sq.unit_end.push_back(p);
+        sq.unit_serial.push_back(serial);
+      }
+      sq.n_eos = sq.n_eot = n_units[b];
+      if (concat && R[b] > 0) sq.concat_off = S[b];
+    }
+    pd.active = ctx->pend[1].active = false;
   } else {
     pd.next_layer = layer + 1;
   }
@@ -868,6 +1045,13 @@ int st_reason_extend(st_ctx *ctx, int32_t layer, const int32_t *seq_ids, const i
                      const int32_t *visible_units, const void *q, const void *k, const void *v, void *out,
                      uint32_t flags, void *stream) {
   return attention_call(ctx, 2, layer, seq_ids, cu_tokens, n_seq, visible_units, q, k, v, out, flags, stream);
+}
+
+int st_forward_packed(st_ctx *ctx, int32_t layer, const int32_t *seq_ids, int32_t n_seq, const int32_t *n_units,
+                      const int32_t *src_unit_len, const int32_t *rsn_unit_len, const int32_t *final_len, int32_t lag_units,
+                      const void *q, const void *k, const void *v, void *out, uint32_t flags, void *stream) {
+  return forward_packed(ctx, layer, seq_ids, n_seq, n_units, src_unit_len, rsn_unit_len, final_len, lag_units, q, k, v, out,
+                        flags, (cudaStream_t)stream);
 }
 
 int st_schedule_build(const int32_t *src_unit_len, const int32_t *rsn_unit_len, int32_t n_units, int32_t final_len,

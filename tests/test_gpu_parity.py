@@ -146,6 +146,52 @@ def test_other_position_modes(position_mode):
         ctx.close()
 
 
+@pytest.mark.parametrize("variant", ["plain", "lag1", "concatenated", "two_term", "simple_kernels"])
+def test_packed_forward_matches_the_oracle_layout(variant):
+    """st_forward_packed: one pass over [source ; reasoning] per sequence under the streaming mask -- the layout the
+    oracle itself materialises -- for ragged schedules (empty units, a sequence without reasoning, several 128-row
+    tiles per unit), every row against the oracle; then three more decode steps continue from the caches it left."""
+    hq = 40 if variant == "two_term" else 32
+    w = workloads.Workload(0, f"packed-{variant}", hq, 8, 1, outlier_frac=0.02 if variant == "two_term" else 0.0,
+                           outlier_mult=8.0 if variant == "two_term" else 1.0)
+    extra = 3
+    scheds = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0),
+              workloads.SeqSchedule((200, 56), (70, 9), 66), workloads.SeqSchedule((130,), (0,), 0)]
+    longer = [workloads.SeqSchedule(s.src_unit_len, s.rsn_unit_len, s.final_len + extra) for s in scheds]
+    lag = 1 if variant == "lag1" else 0
+    pm = api.ST_POS_CONCATENATED if variant == "concatenated" else api.ST_POS_STREAMING
+    total = sum(s.S + s.R for s in scheds)
+    cfg = api.make_config(n_q_heads=hq, n_kv_heads=8, max_batch=len(scheds), n_pages_source=sum((s.S + 63) // 64 for s in scheds),
+                          n_pages_reason=sum((s.R + extra + 63) // 64 for s in scheds), max_tokens_per_call=total,
+                          flags=api.ST_CFG_PRECISE_P if variant == "two_term" else 0, position_mode=pm)
+    ctx = api.Context(cfg)
+    dev = torch.device("cuda", 0)
+    tensors = [workloads.qkv(0, s, b, workload=w) for b, s in enumerate(longer)]
+    q, k, v = (torch.cat([t[i][: s.S + s.R] for t, s in zip(tensors, scheds)]).to(dev) for i in range(3))
+    out = torch.full((total, hq, 128), float("nan"), dtype=torch.float32, device=dev)
+    ids = list(range(len(scheds)))
+    ctx.forward_packed(0, ids, scheds, q, k, v, out, lag_units=lag,
+                       flags=api.ST_REFERENCE_KERNELS if variant == "simple_kernels" else 0)
+    steps = []
+    for i in range(extra):
+        qd, kd, vd = (torch.stack([t[j][s.S + s.R + i] for t, s in zip(tensors, scheds)]).to(dev) for j in range(3))
+        o1 = torch.full((len(scheds), hq, 128), float("nan"), dtype=torch.float32, device=dev)
+        ctx.reason_decode(0, ids, [api.ST_VIS_ALL] * len(scheds), qd, kd, vd, o1)
+        steps.append(o1)
+    torch.cuda.synchronize()
+    ctx.device_status()
+    row = 0
+    for b, (s, sl) in enumerate(zip(scheds, longer)):
+        n = s.S + s.R
+        qb, kb, vb = tensors[b]
+        want = pu.oracle_rows(w, sl, qb, kb, vb, np.arange(sl.S + sl.R), lag_units=lag, position_mode=pm)
+        pu.compare(out[row:row + n].cpu().numpy(), want[:n], f"packed forward {variant} seq {b}")
+        got_steps = torch.stack([o1[b] for o1 in steps]).cpu().numpy()
+        pu.compare(got_steps, want[n:], f"decode steps after the packed forward {variant} seq {b}")
+        row += n
+    ctx.close()
+
+
 def test_page_id_outside_the_pool_is_reported_not_dereferenced():
     """The kernels compare every page id they read with the pool's page count before they build an address from it.
     The test overwrites one entry of the device page table with an id far outside the pool (a host-side test hook,

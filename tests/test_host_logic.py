@@ -316,3 +316,42 @@ def test_a_failing_device_step_rolls_the_call_back():
     assert ctx.reason_decode(0, [0], None, None, None, None, None, check=False) == api.ST_ERR_STATE   # still pending
     ctx.reason_decode(1, [0], None, None, None, None, None)
     assert ctx.seq_state(0)["reason_len"] == 1
+
+
+def test_packed_forward_positions_visibility_and_state():
+    """st_forward_packed on a host-only context: the position ids and visibility of every packed row equal the
+    oracle's schedule (with a lag and with the concatenated ids too), and the sequences end up in the state that
+    streaming the same units would have left."""
+    scheds = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0),
+              workloads.SeqSchedule((), (), 0), workloads.SeqSchedule((7,), (0,), 5)]
+    total = sum(s.S + s.R for s in scheds)
+    for pm, lag in ((api.ST_POS_STREAMING, 0), (api.ST_POS_STREAMING, 1), (api.ST_POS_CONCATENATED, 0)):
+        ctx = host_ctx(n_layers=2, n_pages_source=16, n_pages_reason=8, max_tokens_per_call=total, position_mode=pm)
+        assert ctx.forward_packed(1, [0, 1, 2, 3], scheds, None, None, None, None, check=False) == api.ST_ERR_STATE
+        ctx.forward_packed(0, [0, 1, 2, 3], scheds, None, None, None, None, lag_units=lag)
+        assert ctx.seq_state(0)["source_len"] == 0                                   # not committed before the last layer
+        assert ctx.reason_decode(0, [0], None, None, None, None, None, check=False) == api.ST_ERR_STATE
+        assert ctx.forward_packed(1, [0, 1, 2, 3], scheds, None, None, None, None, lag_units=lag + 1, check=False) == api.ST_ERR_STATE
+        ctx.forward_packed(1, [0, 1, 2, 3], scheds, None, None, None, None, lag_units=lag)
+        pos, vs, vr = ctx.debug_last_call_meta()
+        assert len(pos) == total
+        row = 0
+        for b, s in enumerate(scheds):
+            o = osa.build_schedule(s.src_unit_len, s.rsn_unit_len, s.final_len, lag_units=lag,
+                                   position_mode=POSITION_MODE_NAMES[pm])
+            n = s.S + s.R
+            assert pos[row:row + n].tolist() == o.pos_ids.tolist()
+            assert vs[row:row + s.S].tolist() == list(range(1, s.S + 1)) and vr[row:row + s.S].tolist() == [0] * s.S
+            assert vs[row + s.S:row + n].tolist() == o.vis_len.tolist()
+            assert vr[row + s.S:row + n].tolist() == list(range(1, s.R + 1))
+            st = ctx.seq_state(b)
+            assert st == {"source_len": s.S, "reason_len": s.R, "n_eos": len(s.src_unit_len), "n_eot": len(s.src_unit_len)}
+            row += n
+        # the sequences can be decoded further, and a second packed pass needs them empty
+        ctx.reason_decode(0, [0], [api.ST_VIS_ALL], None, None, None, None)
+        assert ctx.forward_packed(0, [1], scheds[1:2], None, None, None, None, check=False) == api.ST_ERR_STATE
+    ctx = host_ctx(n_pages_source=2, n_pages_reason=8, max_tokens_per_call=total)
+    assert ctx.forward_packed(0, [0], scheds[:1], None, None, None, None, check=False) == api.ST_ERR_OOM_PAGES
+    assert ctx.pages_free() == (2, 8)
+    ctx = host_ctx(n_pages_source=16, n_pages_reason=8, max_tokens_per_call=total, position_mode=api.ST_POS_UNIT_ALIGNED)
+    assert ctx.forward_packed(0, [0], scheds[:1], None, None, None, None, check=False) == api.ST_ERR_INVALID_ARG
