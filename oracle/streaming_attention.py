@@ -26,6 +26,8 @@ a test):
   causal mask that Eq. 2 starts from.
 * RoPE uses the half-split pairing (channel ``c`` with ``c + d/2``) and
   ``inv_freq[c] = theta ** (-2c/d)``.
+* Optional (outside the paper's method, part of its Qwen3 backbones): queries and keys
+  are RMS-normalised per head before the rotation.
 * The caches hold bf16 values, so rotated keys are rounded to bf16
   (round-to-nearest-even) after the fp64 rotation, and rotated queries enter
   the contraction as bf16 too. ``round_rotated=False`` disables both roundings.
@@ -183,6 +185,18 @@ def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
     return np.concatenate([lo * cos - hi * sin, hi * cos + lo * sin], axis=-1)
 
 
+def qk_rmsnorm(x: np.ndarray, weight: np.ndarray, eps: float) -> np.ndarray:
+    """Per-head RMS normalisation of queries or keys over the head dimension, as the Qwen3
+    backbones of Section 4.1 apply it before the rotary embedding:
+    ``x / sqrt(mean(x**2) + eps) * weight`` with ``x [T, H, d]`` and ``weight [d]``."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64).reshape(-1)
+    if w.shape[0] != x.shape[-1]:
+        raise ValueError("one weight per channel of a head is required")
+    ms = (x * x).mean(axis=-1, keepdims=True)
+    return x / np.sqrt(ms + float(eps)) * w
+
+
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Nearest bf16 value (ties to even) of each fp64 element, returned as fp64.
 
@@ -203,8 +217,15 @@ def softmax_rows(z: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------- attention
 
 
-def rotate_and_round(sched: Schedule, q, k, theta: float, round_rotated: bool = True):
-    """Steps 1 and 3: position ids -> RoPE -> the two bf16 rounding points."""
+def rotate_and_round(sched: Schedule, q, k, theta: float, round_rotated: bool = True, qk_norm=None):
+    """Steps 1 and 3: (optional q/k normalisation ->) position ids -> RoPE -> the two bf16 rounding points.
+
+    ``qk_norm = (weight_q, weight_k, eps)`` applies ``qk_rmsnorm`` to q and k first; there is no rounding
+    between the normalisation and the rotation (the fused form: one rounding, after the rotation)."""
+    if qk_norm is not None:
+        wq, wk, eps = qk_norm
+        q = qk_rmsnorm(q, wq, eps)
+        k = qk_rmsnorm(k, wk, eps)
     qh = rope(q, sched.pos_ids, theta)
     kh = rope(k, sched.pos_ids, theta)
     if round_rotated:
@@ -215,7 +236,7 @@ def rotate_and_round(sched: Schedule, q, k, theta: float, round_rotated: bool = 
 
 def attention_rows(sched: Schedule, q, k, v, rows, theta: float = 1.0e6, scale=None,
                    round_rotated: bool = True, row_block: int = 256,
-                   return_probs: bool = False, rotated=None):
+                   return_probs: bool = False, rotated=None, qk_norm=None):
     """Masked softmax attention for the listed rows of ``[source ; reasoning]``.
 
     q: ``[S+R, Hq, d]``; k, v: ``[S+R, Hkv, d]`` (un-rotated, any float dtype).
@@ -236,7 +257,7 @@ def attention_rows(sched: Schedule, q, k, v, rows, theta: float = 1.0e6, scale=N
     s = (1.0 / np.sqrt(d)) if scale is None else float(scale)
     rows = np.asarray(rows, dtype=np.int64).reshape(-1)
 
-    qh, kh = rotated if rotated is not None else rotate_and_round(sched, q, k, theta, round_rotated)
+    qh, kh = rotated if rotated is not None else rotate_and_round(sched, q, k, theta, round_rotated, qk_norm)
 
     O = np.empty((rows.shape[0], Hq, d), dtype=np.float64)
     probs = np.empty((rows.shape[0], Hq, T), dtype=np.float64) if return_probs else None
@@ -253,8 +274,11 @@ def attention_rows(sched: Schedule, q, k, v, rows, theta: float = 1.0e6, scale=N
     return (O, probs) if return_probs else O
 
 
-def expected_cache(sched: Schedule, k, v, theta: float = 1.0e6):
-    """What the two caches must hold: ``bf16(RoPE(k, pos))`` and ``v``, split by stream."""
+def expected_cache(sched: Schedule, k, v, theta: float = 1.0e6, k_norm=None):
+    """What the two caches must hold: ``bf16(RoPE(k, pos))`` and ``v``, split by stream
+    (``k_norm = (weight_k, eps)``: keys normalised first)."""
+    if k_norm is not None:
+        k = qk_rmsnorm(k, k_norm[0], k_norm[1])
     kh = round_to_bf16(rope(k, sched.pos_ids, theta))
     v = np.asarray(v, dtype=np.float64)
     S = sched.S

@@ -252,6 +252,60 @@ def test_position_modes_closed_form():
         osa.build_schedule(n, m, f, position_mode="other")
 
 
+def test_qk_rmsnorm_pins():
+    """The q/k normalisation against scalar loops and torch's rms_norm; with eps = 0 a token's scale cancels, so
+    attention with the normalisation is invariant to rescaling any query or key token; and the whole path with
+    the normalisation equals the scalar brute force fed with rows normalised by the scalar loop."""
+    rng = np.random.default_rng(21)
+    T, H, d = 9, 3, 8
+    x = rng.standard_normal((T, H, d))
+    w = rng.uniform(0.5, 1.5, size=d)
+    eps = 1e-6
+    got = osa.qk_rmsnorm(x, w, eps)
+    want = np.empty_like(x)
+    for t in range(T):
+        for h in range(H):
+            ms = sum(float(x[t, h, c]) ** 2 for c in range(d)) / d
+            for c in range(d):
+                want[t, h, c] = float(x[t, h, c]) / math.sqrt(ms + eps) * float(w[c])
+    assert np.abs(got - want).max() < 1e-14
+    lib = torch.nn.functional.rms_norm(torch.from_numpy(x), (d,), torch.from_numpy(w), eps).numpy()
+    assert np.abs(got - lib).max() < 1e-13
+    ones = osa.qk_rmsnorm(x, np.ones(d), 0.0)
+    assert np.abs((ones ** 2).mean(-1) - 1).max() < 1e-13            # unit weight: every head has RMS 1
+    # scale invariance of the attention rows (eps = 0)
+    n, m, f, Hq, Hkv = [3, 2], [2, 1], 1, 4, 2
+    sched = osa.build_schedule(n, m, f)
+    Tt = sched.S + sched.R
+    q, k, v = rand_qkv(rng, Tt, Hq, Hkv, d, bf16=False)
+    wq, wk = rng.uniform(0.5, 1.5, size=d), rng.uniform(0.5, 1.5, size=d)
+    base = osa.attention_rows(sched, q, k, v, np.arange(Tt), theta=THETA, round_rotated=False, qk_norm=(wq, wk, 0.0))
+    scale = rng.uniform(0.2, 5.0, size=(Tt, 1, 1))
+    scaled = osa.attention_rows(sched, q * scale, k * scale[::-1], v, np.arange(Tt), theta=THETA, round_rotated=False,
+                                qk_norm=(wq, wk, 0.0))
+    assert np.abs(base - scaled).max() < 1e-12
+    plain = osa.attention_rows(sched, q, k, v, np.arange(Tt), theta=THETA, round_rotated=False)
+    assert np.abs(base - plain).max() > 1e-3                         # and it is really applied
+    # brute force on rows normalised by scalar loops (and the cache definition with it)
+    def scalar_norm(a, wv, e):
+        out = np.empty_like(a)
+        for t in range(a.shape[0]):
+            for h in range(a.shape[1]):
+                ms = sum(float(z) ** 2 for z in a[t, h]) / a.shape[2]
+                out[t, h] = [float(z) / math.sqrt(ms + e) * float(g) for z, g in zip(a[t, h], wv)]
+        return out
+    want_rows = brute_force(n, m, f, scalar_norm(q, wq, eps), scalar_norm(k, wk, eps), v, Hq, Hkv, THETA,
+                            round_fn=bf16_via_torch)
+    got_rows = osa.attention_rows(sched, q, k, v, np.arange(Tt), theta=THETA, qk_norm=(wq, wk, eps))
+    assert np.abs(got_rows - want_rows).max() < 1e-12
+    (ks, _), (kr, _) = osa.expected_cache(sched, k, v, THETA, k_norm=(wk, eps))
+    kn = scalar_norm(k, wk, eps)
+    pos = [i if i < sched.S else i - sched.S for i in range(Tt)]
+    want_k = np.array([[[bf16_via_torch(z) for z in scalar_rope(list(kn[i, h]), pos[i], THETA)] for h in range(Hkv)]
+                       for i in range(Tt)])
+    assert np.array_equal(np.concatenate([ks, kr]), want_k)
+
+
 def test_softmax_rows():
     rng = np.random.default_rng(7)
     n, m, f = [3, 4, 2], [2, 3, 1], 3
