@@ -123,6 +123,13 @@ typedef struct st_config {
   int32_t  position_mode;          /* ST_POS_*: position ids of reasoning tokens (source tokens always count
                                       from zero)                                                          */
   int32_t  reserved;               /* must be 0                                                           */
+  const float *q_norm_weight;      /* HOST arrays [n_layers][128], or both NULL: per-head RMS normalisation of */
+  const float *k_norm_weight;      /* q and k over the head dimension before the rotation, x / sqrt(mean(x^2)
+                                      + qk_norm_eps) * weight, as the Qwen3 backbones of Section 4.1 apply it
+                                      (not part of the paper's method; fused into the kernels that rotate:
+                                      one rounding to bf16, after the rotation). Copied at st_create.        */
+  float    qk_norm_eps;            /* e.g. 1e-6                                                             */
+  int32_t  reserved2;              /* must be 0                                                             */
 } st_config;
 
 /* Bytes of device memory the two page pools need: n_layers * (n_pages_source + n_pages_reason) *

@@ -39,6 +39,7 @@ class st_config(C.Structure):
         ("pool_base", C.c_void_p), ("pool_bytes", C.c_uint64),
         ("rope_theta", C.c_double), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
         ("position_mode", C.c_int32), ("reserved", C.c_int32),
+        ("q_norm_weight", C.c_void_p), ("k_norm_weight", C.c_void_p), ("qk_norm_eps", C.c_float), ("reserved2", C.c_int32),
     ]
 
 
@@ -114,10 +115,17 @@ def st_pool_bytes(cfg: st_config) -> int:
 
 def make_config(n_layers=1, n_q_heads=16, n_kv_heads=8, max_batch=1, n_pages_source=0, n_pages_reason=0,
                 max_source_len=0, max_reason_len=0, max_tokens_per_call=1, device=0, pool_base=None, pool_bytes=0,
-                rope_theta=1.0e6, softmax_scale=0.0, flags=0, position_mode=0) -> st_config:
-    return st_config(n_layers, n_q_heads, n_kv_heads, 128, max_batch, 64, n_pages_source, n_pages_reason,
-                     max_source_len, max_reason_len, max_tokens_per_call, device, pool_base, pool_bytes,
-                     rope_theta, softmax_scale, flags, position_mode, 0)
+                rope_theta=1.0e6, softmax_scale=0.0, flags=0, position_mode=0, qk_norm=None) -> st_config:
+    """qk_norm: (weight_q, weight_k, eps) with float32 numpy arrays [n_layers, 128] (host), or None."""
+    cfg = st_config(n_layers, n_q_heads, n_kv_heads, 128, max_batch, 64, n_pages_source, n_pages_reason,
+                    max_source_len, max_reason_len, max_tokens_per_call, device, pool_base, pool_bytes,
+                    rope_theta, softmax_scale, flags, position_mode, 0, None, None, 0.0, 0)
+    if qk_norm is not None:
+        wq = np.ascontiguousarray(qk_norm[0], dtype=np.float32).reshape(n_layers, 128)
+        wk = np.ascontiguousarray(qk_norm[1], dtype=np.float32).reshape(n_layers, 128)
+        cfg._keep = (wq, wk)                       # the library copies them in st_create; keep them alive until then
+        cfg.q_norm_weight, cfg.k_norm_weight, cfg.qk_norm_eps = wq.ctypes.data, wk.ctypes.data, float(qk_norm[2])
+    return cfg
 
 
 class Context:

@@ -74,6 +74,7 @@ struct st_ctx {
   __nv_bfloat16 *qhat[2] = {nullptr, nullptr};  // rotated-query scratch per side
   float *partial = nullptr;                     // split-K workspace (reasoning side)
   double2 *rope_hi = nullptr, *rope_lo = nullptr;   // rotation tables of the fused decode append
+  float *d_norm = nullptr;                          // q/k normalisation weights [layer][q, k][128], or nullptr
   int32_t *d_status = nullptr;
   // staging for ST_IO_HOST, per side
   __nv_bfloat16 *stage_q[2] = {nullptr, nullptr}, *stage_k[2] = {nullptr, nullptr}, *stage_v[2] = {nullptr, nullptr};
@@ -140,7 +141,9 @@ bool config_ok(const st_config *c, std::string *why) {
   if (!(c->rope_theta > 0.0)) return bad("rope_theta must be > 0");
   if (c->softmax_scale < 0.f) return bad("softmax_scale must be >= 0");
   if (c->position_mode < ST_POS_STREAMING || c->position_mode > ST_POS_UNIT_ALIGNED) return bad("unknown position_mode");
-  if (c->reserved != 0) return bad("reserved must be 0");
+  if (c->reserved != 0 || c->reserved2 != 0) return bad("reserved fields must be 0");
+  if ((c->q_norm_weight == nullptr) != (c->k_norm_weight == nullptr)) return bad("q_norm_weight and k_norm_weight go together");
+  if (c->q_norm_weight && !(c->qk_norm_eps >= 0.f)) return bad("qk_norm_eps must be >= 0");
   return true;
 }
 
@@ -170,6 +173,7 @@ void release_device(st_ctx *ctx) {
   cudaFree(ctx->partial);
   cudaFree(ctx->rope_hi);
   cudaFree(ctx->rope_lo);
+  cudaFree(ctx->d_norm);
   cudaFree(ctx->d_status);
   if (ctx->own_pool) cudaFree(ctx->pool_alloc);
 }
@@ -465,6 +469,9 @@ int run_append(st_ctx *ctx, int which, int32_t layer, const int32_t *seq_ids, co
     ap.ptab_stride = ctx->ptab_stride[which];
     ap.n_pages = (int32_t)(which ? ctx->cfg.n_pages_reason : ctx->cfg.n_pages_source);
     ap.status = ctx->d_status;
+    ap.norm_q = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 : nullptr;
+    ap.norm_k = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 + 128 : nullptr;
+    ap.norm_eps = ctx->cfg.qk_norm_eps;
     ap.n_seq = ns;
     ap.n_q_heads = ctx->cfg.n_q_heads;
     ap.n_kv_heads = ctx->cfg.n_kv_heads;
@@ -506,6 +513,9 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
   p->group = ctx->group;
   p->scale_log2 = ctx->scale_log2;
   memcpy(p->inv_freq, ctx->inv_freq, sizeof(p->inv_freq));
+  p->norm_q = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 : nullptr;
+  p->norm_k = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 + 128 : nullptr;
+  p->norm_eps = ctx->cfg.qk_norm_eps;
   p->total_work = p->work_per_cta = p->n_cta = 0;
 }
 
@@ -972,6 +982,16 @@ int st_create(const st_config *cfg, st_ctx **out) {
       ST_CREATE_CUDA(st::launch_rope_table(ctx->inv_freq, ctx->rope_hi, n_hi, st::kRopeLoSteps, nullptr));
       ST_CREATE_CUDA(st::launch_rope_table(ctx->inv_freq, ctx->rope_lo, st::kRopeLoSteps, 1, nullptr));
     }
+    if (cfg->q_norm_weight) {
+      std::vector<float> w((size_t)cfg->n_layers * 256);
+      for (int l = 0; l < cfg->n_layers; ++l) {
+        std::copy_n(cfg->q_norm_weight + (size_t)l * 128, 128, w.begin() + (size_t)l * 256);
+        std::copy_n(cfg->k_norm_weight + (size_t)l * 128, 128, w.begin() + (size_t)l * 256 + 128);
+      }
+      ST_CREATE_CUDA(cudaMalloc(&ctx->d_norm, sizeof(float) * w.size()));
+      ST_CREATE_CUDA(cudaMemcpy(ctx->d_norm, w.data(), sizeof(float) * w.size(), cudaMemcpyHostToDevice));
+    }
+    ctx->cfg.q_norm_weight = ctx->cfg.k_norm_weight = nullptr;   // (the caller's arrays are not used after this call)
     ST_CREATE_CUDA(cudaMalloc(&ctx->d_status, sizeof(int32_t)));
     ST_CREATE_CUDA(cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
     ST_CREATE_CUDA(cudaDeviceSynchronize());

@@ -390,7 +390,12 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         const int r_end = min(r_lo + kRowsPerTile, packed_rows);
         const int tok_lo = div_g(r_lo), tok_hi = div_g(r_end - 1);
         const int n_items = (tok_hi - tok_lo + 1) * 8;
-        for (int it = r_local; it < n_items; it += kRowsPerTile) {
+        const bool norm = p.norm_q != nullptr;
+        for (int base = 0; base < n_items; base += kRowsPerTile) {
+          // (the 8 items of a token sit in 8 neighbouring lanes: all of them are in range or none)
+          const int it = base + r_local;
+          const unsigned lanes = __ballot_sync(0xffffffffu, it < n_items);
+          if (it >= n_items) continue;
           const int tk = tok_lo + (it >> 3), c = it & 7;
           float cs[8], sn[8];
           const double pos = (double)(sq.b_base + tk + sq.rope_off);
@@ -416,15 +421,38 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
 #pragma unroll
           for (int g = 0; g < kMaxGroup; ++g) {
             const int rr = tk * G + g - r_lo;
-            if (g < G && rr >= 0 && rr < r_end - r_lo) {
+            const bool valid = g < G && rr >= 0 && rr < r_end - r_lo;
+            const unsigned row_lanes = __ballot_sync(lanes, valid);   // the lanes that take part in this row's shuffles
+            if (valid) {
               const uint32_t *lo_w = reinterpret_cast<const uint32_t *>(&lo_raw[g]);
               const uint32_t *hi_w = reinterpret_cast<const uint32_t *>(&hi_raw[g]);
               uint32_t lo_out[4], hi_out[4];
+              // optional RMS normalisation of the row over its 128 channels: the 8 lanes of the token add their squares
+              float rs = 1.f;
+              if (norm) {
+                float ss = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float a0 = __uint_as_float(lo_w[e] << 16), a1 = __uint_as_float(lo_w[e] & 0xffff0000u);
+                  const float b0 = __uint_as_float(hi_w[e] << 16), b1 = __uint_as_float(hi_w[e] & 0xffff0000u);
+                  ss += a0 * a0 + a1 * a1 + b0 * b0 + b1 * b1;
+                }
+                ss += __shfl_xor_sync(row_lanes, ss, 1);
+                ss += __shfl_xor_sync(row_lanes, ss, 2);
+                ss += __shfl_xor_sync(row_lanes, ss, 4);
+                rs = rsqrtf(ss * (1.f / kHeadDim) + p.norm_eps);
+              }
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 // two channels per word: x = channels 8c+2e, 8c+2e+1, y = their partners 64 channels on
-                const float2 x = make_float2(__uint_as_float(lo_w[e] << 16), __uint_as_float(lo_w[e] & 0xffff0000u));
-                const float2 y = make_float2(__uint_as_float(hi_w[e] << 16), __uint_as_float(hi_w[e] & 0xffff0000u));
+                float2 x = make_float2(__uint_as_float(lo_w[e] << 16), __uint_as_float(lo_w[e] & 0xffff0000u));
+                float2 y = make_float2(__uint_as_float(hi_w[e] << 16), __uint_as_float(hi_w[e] & 0xffff0000u));
+                if (norm) {
+                  x.x *= rs * p.norm_q[8 * c + 2 * e];
+                  x.y *= rs * p.norm_q[8 * c + 2 * e + 1];
+                  y.x *= rs * p.norm_q[64 + 8 * c + 2 * e];
+                  y.y *= rs * p.norm_q[64 + 8 * c + 2 * e + 1];
+                }
                 const float2 c2 = make_float2(cs[2 * e], cs[2 * e + 1]), s2 = make_float2(sn[2 * e], sn[2 * e + 1]);
                 const float2 ns2 = make_float2(-sn[2 * e], -sn[2 * e + 1]);
                 const float2 lo_r = ffma2(x, c2, fmul2(y, ns2));          // x cos - y sin

@@ -68,7 +68,13 @@ __global__ void __launch_bounds__(256) st_k_rope_append(const __grid_constant__ 
   // keys and queries: one item = (token, head, pair of 16-byte chunks c and c + 64)
   const int items_k = nt * Hkv * 8;
   const int items_q = (p.qhat != nullptr) ? nt * Hq * 8 : 0;
-  for (int it = threadIdx.x; it < items_k + items_q; it += blockDim.x) {
+  const bool norm = p.norm_k != nullptr;
+  for (int base = 0; base < items_k + items_q; base += blockDim.x) {
+    // (the 8 items of one (token, head) row sit in 8 neighbouring lanes: either all of them are in range or none)
+    const int it = base + threadIdx.x;
+    const bool in_range = it < items_k + items_q;
+    const unsigned lanes = __ballot_sync(0xffffffffu, in_range);
+    if (!in_range) continue;
     const bool is_q = it >= items_k;
     const int j = is_q ? it - items_k : it;
     const int H = is_q ? Hq : Hkv;
@@ -83,10 +89,29 @@ __global__ void __launch_bounds__(256) st_k_rope_append(const __grid_constant__ 
     uint4 lo_out, hi_out;
     __nv_bfloat16 *lo_o = reinterpret_cast<__nv_bfloat16 *>(&lo_out);
     __nv_bfloat16 *hi_o = reinterpret_cast<__nv_bfloat16 *>(&hi_out);
+    // optional RMS normalisation of the row over its 128 channels, in fp64 like the rotation: x / sqrt(mean(x^2) + eps) * w
+    double rs = 1.0;
+    const float *nw = is_q ? p.norm_q : p.norm_k;
+    if (norm) {
+      double ss = 0.0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const double x = (double)__bfloat162float(lo[e]), y = (double)__bfloat162float(hi[e]);
+        ss += x * x + y * y;
+      }
+      ss += __shfl_xor_sync(lanes, ss, 1);
+      ss += __shfl_xor_sync(lanes, ss, 2);
+      ss += __shfl_xor_sync(lanes, ss, 4);
+      rs = 1.0 / sqrt(ss * (1.0 / kHeadDim) + (double)p.norm_eps);
+    }
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       const double cs = s_cos[t][8 * cp + e], sn = s_sin[t][8 * cp + e];
-      const double x = (double)__bfloat162float(lo[e]), y = (double)__bfloat162float(hi[e]);
+      double x = (double)__bfloat162float(lo[e]), y = (double)__bfloat162float(hi[e]);
+      if (norm) {
+        x = x * rs * (double)nw[8 * cp + e];
+        y = y * rs * (double)nw[64 + 8 * cp + e];
+      }
       lo_o[e] = __double2bfloat16(x * cs - y * sn);
       hi_o[e] = __double2bfloat16(y * cs + x * sn);
     }

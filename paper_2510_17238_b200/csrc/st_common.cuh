@@ -68,6 +68,9 @@ struct AppendParams {
   int32_t ptab_stride;
   int32_t n_pages;                 // pages of the pool: a page id outside [0, n_pages) is reported, not used
   int32_t *status;                 // device status word
+  // per-head RMS normalisation of q and k before the rotation (nullptr: none): weights of this layer, [128] each
+  const float *norm_q, *norm_k;
+  float norm_eps;
   int32_t n_seq, n_q_heads, n_kv_heads;
   double inv_freq[64];             // theta^(-2c/128), c = 0..63
   AppendSeq seq[kMaxSeqPerLaunch];
@@ -106,6 +109,9 @@ struct AttnParams {
   int32_t n_cta;
   float scale_log2;                // softmax scale * log2(e)
   double inv_freq[64];             // theta^(-2c/128): the tensor-core kernel rotates its queries itself (from q_raw)
+  // per-head RMS normalisation of q and k before the rotation, for the kernels that rotate their own (nullptr: none)
+  const float *norm_q, *norm_k;
+  float norm_eps;
   // decode with the append fused in: (cos, sin) of k * 1024 * inv_freq[c] and of j * inv_freq[c], j < 1024, as [.][64]
   const double2 *rope_hi, *rope_lo;
   AttnSeq seq[kMaxSeqPerLaunch];

@@ -242,6 +242,30 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
 #pragma unroll
           for (int i = 0; i < 4; ++i) vv[i] = vsrc[lane + 32 * i];
         }
+        // optional RMS normalisation of the query rows and of the new key over their 128 channels (fp64, as in the
+        // append kernel): every lane holds 4 channels of a row, the warp adds the squares
+        const bool norm = p.norm_k != nullptr;
+        double wq[2][2] = {{1.0, 1.0}, {1.0, 1.0}}, wk[2][2] = {{1.0, 1.0}, {1.0, 1.0}};   // [i][low/high half]
+        if (norm) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            wq[i][0] = (double)p.norm_q[lane + 32 * i];
+            wq[i][1] = (double)p.norm_q[lane + 32 * i + 64];
+            wk[i][0] = (double)p.norm_k[lane + 32 * i];
+            wk[i][1] = (double)p.norm_k[lane + 32 * i + 64];
+          }
+        }
+        auto row_scale = [&](const __nv_bfloat16 (&x)[2], const __nv_bfloat16 (&y)[2]) -> double {
+          double ss = 0.0;
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const double a = (double)__bfloat162float(x[i]), b = (double)__bfloat162float(y[i]);
+            ss += a * a + b * b;
+          }
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+          return 1.0 / sqrt(ss * (1.0 / kHeadDim) + (double)p.norm_eps);
+        };
         double cs[2], sn[2];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {              // angle addition from the two rotation tables
@@ -251,10 +275,15 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           if (g < G) {
+            const double rs = norm ? row_scale(qx[g], qy[g]) : 1.0;
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               const int c = lane + 32 * i;
-              const double x = (double)__bfloat162float(qx[g][i]), y = (double)__bfloat162float(qy[g][i]);
+              double x = (double)__bfloat162float(qx[g][i]), y = (double)__bfloat162float(qy[g][i]);
+              if (norm) {
+                x = x * rs * wq[i][0];
+                y = y * rs * wq[i][1];
+              }
               sm.qhat[slot][g][c] = __double2bfloat16(x * cs[i] - y * sn[i]);
               sm.qhat[slot][g][c + 64] = __double2bfloat16(y * cs[i] + x * sn[i]);
             }
@@ -266,10 +295,15 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         if (owns_last) {
           uint8_t *blk = const_cast<uint8_t *>(p.pool_b) + ((size_t)page * Hkv + kvh) * kBlockBytes;
           const int tok = pos & 63;
+          const double rs = norm ? row_scale(kx, ky) : 1.0;
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
             const int c = lane + 32 * i;
-            const double x = (double)__bfloat162float(kx[i]), y = (double)__bfloat162float(ky[i]);
+            double x = (double)__bfloat162float(kx[i]), y = (double)__bfloat162float(ky[i]);
+            if (norm) {
+              x = x * rs * wk[i][0];
+              y = y * rs * wk[i][1];
+            }
             *reinterpret_cast<__nv_bfloat16 *>(blk + k_byte_offset(tok, c)) = __double2bfloat16(x * cs[i] - y * sn[i]);
             *reinterpret_cast<__nv_bfloat16 *>(blk + k_byte_offset(tok, c + 64)) = __double2bfloat16(y * cs[i] + x * sn[i]);
           }

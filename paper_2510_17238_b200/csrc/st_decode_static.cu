@@ -126,6 +126,7 @@ extern "C" int st_decode_attention_static(int32_t device, const void *pool_sourc
   p.ptab_b = page_table_reason;
   p.ptab_stride_a = table_stride_source;
   p.ptab_stride_b = table_stride_reason;
+  p.norm_q = p.norm_k = nullptr;
   p.n_pages_a = (int32_t)n_pages_source;
   p.n_pages_b = (int32_t)n_pages_reason;
   p.qhat = (const __nv_bfloat16 *)q_rotated;

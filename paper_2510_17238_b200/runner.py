@@ -147,7 +147,7 @@ def pool_pages(scheds):
 
 
 def make_context(workload, scheds, plan: Plan, n_layers=None, device=0, extra_pages=0, flags=0,
-                 position_mode=0) -> api.Context:
+                 position_mode=0, qk_norm=None) -> api.Context:
     ps, pr = pool_pages(scheds)
     cfg = api.make_config(
         n_layers=workload.n_layers if n_layers is None else n_layers,
@@ -155,7 +155,7 @@ def make_context(workload, scheds, plan: Plan, n_layers=None, device=0, extra_pa
         n_pages_source=ps + extra_pages, n_pages_reason=pr + extra_pages,
         max_source_len=max(s.S for s in scheds), max_reason_len=max(max(s.R for s in scheds), 1),
         max_tokens_per_call=plan.max_call_tokens, device=device, rope_theta=workload.rope_theta, flags=flags,
-        position_mode=position_mode)
+        position_mode=position_mode, qk_norm=qk_norm)
     return api.Context(cfg)
 
 

@@ -12,12 +12,12 @@ REL_L2_TOL = 5e-3
 POSITION_MODE_NAMES = {0: "streaming", 1: "concatenated", 2: "unit_aligned"}
 
 
-def oracle_rows(workload, sched, q, k, v, rows, lag_units=0, position_mode=0):
+def oracle_rows(workload, sched, q, k, v, rows, lag_units=0, position_mode=0, qk_norm=None):
     """fp64 oracle outputs for the listed rows of one sequence (q/k/v: CPU bf16 [S+R, H, 128])."""
     o = osa.build_schedule(sched.src_unit_len, sched.rsn_unit_len, sched.final_len, lag_units=lag_units,
                            position_mode=POSITION_MODE_NAMES[position_mode])
     return osa.attention_rows(o, q.double().numpy(), k.double().numpy(), v.double().numpy(), rows,
-                              theta=workload.rope_theta)
+                              theta=workload.rope_theta, qk_norm=qk_norm)
 
 
 def sample_rows(sched, n_random, seed):
@@ -56,11 +56,12 @@ def compare(got, want, what=""):
 
 
 def run_plan(workload, scheds, index, mode="decode", lookahead=1, two_streams=False, extra_flags=0, layer_seeds=(0,),
-             flat_inputs=None, n_layers=None, lag_units=0, cfg_flags=0, position_mode=0):
+             flat_inputs=None, n_layers=None, lag_units=0, cfg_flags=0, position_mode=0, qk_norm=None):
     """Runs a whole plan on the GPU. Returns (ctx, plan, batches, flats) with outputs synchronised."""
     plan = runner.make_plan(scheds, mode=mode, lookahead=lookahead, lag_units=lag_units)
     L = len(layer_seeds) if n_layers is None else n_layers
-    ctx = runner.make_context(workload, scheds, plan, n_layers=L, flags=cfg_flags, position_mode=position_mode)
+    ctx = runner.make_context(workload, scheds, plan, n_layers=L, flags=cfg_flags, position_mode=position_mode,
+                              qk_norm=qk_norm)
     flats, batches = [], []
     for layer in range(L):
         fl = flat_inputs[layer] if flat_inputs is not None else runner.flatten_inputs(
@@ -80,7 +81,7 @@ def run_plan(workload, scheds, index, mode="decode", lookahead=1, two_streams=Fa
 
 
 def check_against_oracle(workload, scheds, plan, batch, flat, n_random=None, full_seqs=(), what="", lag_units=0,
-                         position_mode=0):
+                         position_mode=0, qk_norm=None):
     """Compares a layer's GPU outputs with the oracle: all rows for `full_seqs` (or every sequence when
     n_random is None), unit-boundary rows plus n_random seeded rows otherwise."""
     out = batch.outputs_flat()
@@ -92,7 +93,7 @@ def check_against_oracle(workload, scheds, plan, batch, flat, n_random=None, ful
             continue
         rows = np.arange(hi - lo) if (n_random is None or b in full_seqs) else sample_rows(s, n_random, b)
         want = oracle_rows(workload, s, fq[lo:hi], fk[lo:hi], fv[lo:hi], rows, lag_units=lag_units,
-                           position_mode=position_mode)
+                           position_mode=position_mode, qk_norm=qk_norm)
         got = out[lo:hi][torch.from_numpy(rows)].numpy()
         r = compare(got, want, f"{what} seq {b}")
         worst = (max(worst[0], r[0]), max(worst[1], r[1]))
@@ -101,7 +102,7 @@ def check_against_oracle(workload, scheds, plan, batch, flat, n_random=None, ful
     return worst
 
 
-def check_cache(ctx, workload, scheds, plan, flat, layer=0, seqs=None, position_mode=0):
+def check_cache(ctx, workload, scheds, plan, flat, layer=0, seqs=None, position_mode=0, k_norm=None):
     """Cache contents vs the oracle's definition bf16(RoPE_fp64(k)), v. Returns mismatching key elements."""
     fq, fk, fv = flat
     bad = 0
@@ -111,7 +112,7 @@ def check_cache(ctx, workload, scheds, plan, flat, layer=0, seqs=None, position_
         lo, hi = int(plan.seq_offset[b]), int(plan.seq_offset[b + 1])
         o = osa.build_schedule(s.src_unit_len, s.rsn_unit_len, s.final_len, position_mode=POSITION_MODE_NAMES[position_mode])
         (ks, vs), (kr, vr) = osa.expected_cache(o, fk[lo:hi].double().numpy(), fv[lo:hi].double().numpy(),
-                                                workload.rope_theta)
+                                                workload.rope_theta, k_norm=k_norm)
         for which, (kw, vw, n) in enumerate(((ks, vs, s.S), (kr, vr, s.R))):
             if n == 0:
                 continue

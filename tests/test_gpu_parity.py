@@ -192,6 +192,31 @@ def test_packed_forward_matches_the_oracle_layout(variant):
     ctx.close()
 
 
+@pytest.mark.parametrize("two_term", [False, True])
+def test_qk_rmsnorm_fused_into_the_rotating_kernels(two_term):
+    """Per-head RMS normalisation of q and k (Qwen3) in front of the rotation, in every kernel that rotates: the
+    append kernel (keys of chunks and spans, queries of the two-term variant), the decode kernel's fused append (new
+    key and the step's queries) and the attention kernel's query rotation. Two layers with different weights; rows
+    of both layers and the caches (normalised, rotated, rounded once) against the oracle."""
+    w = small_workload(40)
+    rng = np.random.default_rng(33)
+    wq = rng.uniform(0.5, 1.5, size=(2, 128)).astype(np.float32)
+    wk = rng.uniform(0.5, 1.5, size=(2, 128)).astype(np.float32)
+    eps = 1e-6
+    scheds = [workloads.SeqSchedule((30, 70, 64, 5), (3, 2, 4, 2), 3), workloads.SeqSchedule((64, 1, 129), (2, 0, 3), 0),
+              workloads.SeqSchedule((200, 56), (70, 9), 66)]
+    flags = api.ST_CFG_PRECISE_P if two_term else 0
+    for mode in ("decode", "extend"):
+        ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode=mode, lookahead=2, layer_seeds=(0, 1), cfg_flags=flags,
+                                                qk_norm=(wq, wk, eps))
+        for layer in range(2):
+            norm = (wq[layer], wk[layer], eps)
+            pu.check_against_oracle(w, scheds, plan, batches[layer], flats[layer], what=f"qk norm {mode} layer {layer}",
+                                    qk_norm=norm)
+            assert pu.check_cache(ctx, w, scheds, plan, flats[layer], layer=layer, k_norm=(wk[layer], eps)) <= 2
+        ctx.close()
+
+
 def test_page_id_outside_the_pool_is_reported_not_dereferenced():
     """The kernels compare every page id they read with the pool's page count before they build an address from it.
     The test overwrites one entry of the device page table with an id far outside the pool (a host-side test hook,
