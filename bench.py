@@ -60,6 +60,9 @@ def parse_args():
     ap.add_argument("--spans", action="store_true",
                     help="side measurement: reasoning units and the final stage teacher-forced as spans "
                          "(st_reason_extend) on one stream; prints its own JSON line")
+    ap.add_argument("--arrival", action="store_true",
+                    help="side measurement: batch / interleaved / streaming routes under the paper's input arrival "
+                         "process (150 words per minute); prints its own JSON line")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the compact measurements of workloads 4 and 3 that the default run appends as per_config")
@@ -238,6 +241,85 @@ def run_spans(args, w, scheds, local_rank):
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tflops / peaks["bf16_tflops"],
                      "of": peaks["source"], "launches": n_tc, "total_ms": ms_tc, "traffic": None}}))
     ctx.close()
+
+
+def run_arrival(args, local_rank):
+    """Side measurement (--arrival): the three attention routes of Section 3.3 under the paper's input arrival process
+    (150 words per minute). One sequence shaped like the paper's GSM-Symbolic samples (Table 4: about 5 input units,
+    about 440 reasoning tokens), Qwen3-4B heads; every library call is timed on the device (CUDA events), and the
+    timeline of each route is computed from those durations (paper_2510_17238_b200/arrival.py): attention only
+    (x 36 layers), and with the paper's own full-model call times (Table 4: 0.041 s per prefill, 0.037 s per decode
+    step) added, which is what its latency tables contain."""
+    from paper_2510_17238_b200 import api, arrival, workloads
+    n_units, n_src, n_rsn, final = 5, 20, 80, 40
+    sched = workloads.SeqSchedule((n_src,) * n_units, (n_rsn,) * n_units, final)
+    w = workloads.Workload(2, "arrival-qwen3-4b-b1-5x(20,80)+40", 32, 8, 1)
+    dev = torch.device("cuda", local_rank)
+    q, k, v = (t.to(dev) for t in workloads.qkv(2, sched, 0, workload=w))
+    S, R = sched.S, sched.R
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def timed_call(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3
+
+    def one_pass(batch_route):
+        cfg = api.make_config(n_q_heads=32, n_kv_heads=8, max_batch=1, n_pages_source=S // 64 + 2, n_pages_reason=R // 64 + 2,
+                              max_tokens_per_call=max(S, 128),
+                              position_mode=api.ST_POS_CONCATENATED if batch_route else api.ST_POS_STREAMING)
+        ctx = api.Context(cfg)
+        out = torch.empty((max(S, 128), 32, 128), dtype=torch.float32, device=dev)
+        pre, dec = [], []
+        if batch_route:
+            pre.append(timed_call(lambda: ctx.append_source_chunk(0, [0], [0, S], q[:S], k[:S], v[:S], out, api.ST_END_OF_UNIT, stream)))
+        r = 0
+        for u in range(n_units):
+            if not batch_route:
+                sl = slice(u * n_src, (u + 1) * n_src)
+                pre.append(timed_call(lambda: ctx.append_source_chunk(0, [0], [0, n_src], q[sl], k[sl], v[sl], out, api.ST_END_OF_UNIT, stream)))
+            for i in range(n_rsn):
+                sl = slice(S + r, S + r + 1)
+                vis = [api.ST_VIS_ALL] if batch_route else None
+                flags = api.ST_END_OF_UNIT if (i == n_rsn - 1 and not batch_route) else 0
+                dec.append(timed_call(lambda: ctx.reason_decode(0, [0], vis, q[sl], k[sl], v[sl], out, flags, stream)))
+                r += 1
+        for i in range(final):
+            sl = slice(S + r, S + r + 1)
+            dec.append(timed_call(lambda: ctx.reason_decode(0, [0], [api.ST_VIS_ALL], q[sl], k[sl], v[sl], out, 0, stream)))
+            r += 1
+        ctx.device_status()
+        ctx.close()
+        return pre, dec
+
+    for _ in range(max(1, args.warmup)):
+        one_pass(False)
+    pre_s, dec_s = one_pass(False)
+    pre_b, dec_b = one_pass(True)
+    layers = 36
+    routes = {}
+    for label, extra_pre, extra_dec in (("attention_only_x36_layers", 0.0, 0.0), ("with_paper_full_model_call_times", 0.041, 0.037)):
+        rows = {}
+        for route in ("batch", "interleaved", "streaming"):
+            pre, dec = (pre_b, dec_b) if route == "batch" else (pre_s, dec_s)
+            tl = arrival.simulate(route, sched.src_unit_len, sched.rsn_unit_len, sched.final_len,
+                                  lambda u, n: layers * pre[min(u, len(pre) - 1)] + extra_pre,
+                                  lambda r: layers * dec[r] + extra_dec)
+            rows[route] = {"ttft_tokens": tl.ttft_tokens, "first_reasoning_token_s": tl.first_token_s,
+                           "input_end_s": tl.input_end_s, "delay_after_input_s": tl.delay_s}
+        routes[label] = rows
+    print(json.dumps({
+        "metric": "time to the first reasoning token and delay after the end of the input, three attention routes, input at 150 words/min",
+        "config": {"workload": w.name, "units": n_units, "source_tokens": S, "reasoning_tokens": R, "layers_assumed": layers,
+                   "tokens_per_word": arrival.TOKENS_PER_WORD},
+        "measured_call_us": {"prefill_unit_mean": 1e6 * statistics.mean(pre_s), "prefill_all_input": 1e6 * pre_b[0],
+                             "decode_step_mean": 1e6 * statistics.mean(dec_s)},
+        "routes": routes, "data": "synthetic",
+        "note": "paper, Table 2 (GSM-Symbolic, Qwen3-4B): tokens before reasoning 94.74 (batch) -> 20.77 (streaming); "
+                "Table 4: first-token latency 28.0 s -> 6.2 s; other hardware, context only"}))
 
 
 def oracle_sample(index, scheds, w, rows_per_sample, seed=0):
@@ -506,6 +588,10 @@ def main():
     if args.spans:
         if rank == 0:
             run_spans(args, w, scheds, local_rank)
+        return
+    if args.arrival:
+        if rank == 0:
+            run_arrival(args, local_rank)
         return
 
     plan = runner.make_plan(scheds, mode="decode", lookahead=1)
