@@ -271,7 +271,10 @@ __device__ __forceinline__ void add_bf16x2(float &acc_lo, float &acc_hi, uint32_
 // kPrecise: the probabilities enter P V as two bf16 terms (p = hi + lo, 16 significant bits) instead of one. One bf16
 // term bounds a row's error by about 2^-9 times the largest |v| it mixes, which leaves the 1e-2 tolerance when values
 // reach a few tens (outlier channels); the second term costs one more P V product per key tile.
-template <bool kPrecise>
+// kNorm (one-term variant only): per-head RMS normalisation of the query rows in front of their rotation. A template
+// parameter because the same code as a run-time option cost the kernel 6 us per launch with the option off (788 against
+// 820 TFLOP/s on the appends of the benchmark workload).
+template <bool kPrecise, bool kNorm>
 __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constant__ AttnParams p) {
   constexpr int kKStages = kPrecise ? 1 : kKStagesFast;
   extern __shared__ uint8_t smem_raw[];
@@ -390,12 +393,15 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         const int r_end = min(r_lo + kRowsPerTile, packed_rows);
         const int tok_lo = div_g(r_lo), tok_hi = div_g(r_end - 1);
         const int n_items = (tok_hi - tok_lo + 1) * 8;
-        const bool norm = p.norm_q != nullptr;
-        for (int base = 0; base < n_items; base += kRowsPerTile) {
-          // (the 8 items of a token sit in 8 neighbouring lanes: all of them are in range or none)
-          const int it = base + r_local;
-          const unsigned lanes = __ballot_sync(0xffffffffu, it < n_items);
-          if (it >= n_items) continue;
+        constexpr bool norm = kNorm;
+        // (with the normalisation the whole warp walks the loop together, for the shuffles: the 8 items of a token sit
+        // in 8 neighbouring lanes, all of them in range or none)
+        for (int it = r_local; kNorm ? it - r_local < n_items : it < n_items; it += kRowsPerTile) {
+          unsigned lanes = 0xffffffffu;
+          if constexpr (kNorm) {
+            lanes = __ballot_sync(0xffffffffu, it < n_items);
+            if (it >= n_items) continue;
+          }
           const int tk = tok_lo + (it >> 3), c = it & 7;
           float cs[8], sn[8];
           const double pos = (double)(sq.b_base + tk + sq.rope_off);
@@ -422,14 +428,15 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           for (int g = 0; g < kMaxGroup; ++g) {
             const int rr = tk * G + g - r_lo;
             const bool valid = g < G && rr >= 0 && rr < r_end - r_lo;
-            const unsigned row_lanes = __ballot_sync(lanes, valid);   // the lanes that take part in this row's shuffles
+            unsigned row_lanes = 0u;
+            if constexpr (kNorm) row_lanes = __ballot_sync(lanes, valid);   // the lanes that take part in this row's shuffles
             if (valid) {
               const uint32_t *lo_w = reinterpret_cast<const uint32_t *>(&lo_raw[g]);
               const uint32_t *hi_w = reinterpret_cast<const uint32_t *>(&hi_raw[g]);
               uint32_t lo_out[4], hi_out[4];
               // optional RMS normalisation of the row over its 128 channels: the 8 lanes of the token add their squares
               float rs = 1.f;
-              if (norm) {
+              if constexpr (norm) {
                 float ss = 0.f;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -447,7 +454,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
                 // two channels per word: x = channels 8c+2e, 8c+2e+1, y = their partners 64 channels on
                 float2 x = make_float2(__uint_as_float(lo_w[e] << 16), __uint_as_float(lo_w[e] & 0xffff0000u));
                 float2 y = make_float2(__uint_as_float(hi_w[e] << 16), __uint_as_float(hi_w[e] & 0xffff0000u));
-                if (norm) {
+                if constexpr (norm) {
                   x.x *= rs * p.norm_q[8 * c + 2 * e];
                   x.y *= rs * p.norm_q[8 * c + 2 * e + 1];
                   y.x *= rs * p.norm_q[64 + 8 * c + 2 * e];
@@ -794,9 +801,11 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
 }
 
 cudaError_t init_attn_tc_kernels() {
-  cudaError_t e = cudaFuncSetAttribute(st_k_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
+  cudaError_t e = cudaFuncSetAttribute(st_k_attn_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(st_k_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
+  e = cudaFuncSetAttribute(st_k_attn_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(st_k_attn_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024);
 }
 
 int attn_tc_rows_per_cta() { return kRowsPerCta; }
@@ -814,8 +823,9 @@ cudaError_t launch_attn_tc(AttnParams &p, bool precise, int num_sms, cudaStream_
   p.total_work = total;
   p.n_cta = total;
   if (t0) cudaEventRecord(t0, stream);
-  cudaError_t e = launch_dependent(precise ? st_k_attn_tc<true> : st_k_attn_tc<false>, dim3(total), dim3(kThreads),
-                                   kSmemBytes + 1024, stream, p);
+  // (the two-term variant takes queries that the append kernel has normalised and rotated)
+  auto kernel = precise ? st_k_attn_tc<true, false> : p.norm_q != nullptr ? st_k_attn_tc<false, true> : st_k_attn_tc<false, false>;
+  cudaError_t e = launch_dependent(kernel, dim3(total), dim3(kThreads), kSmemBytes + 1024, stream, p);
   if (e != cudaSuccess) return e;
   if (t1) cudaEventRecord(t1, stream);
   *n_launches = 1;
