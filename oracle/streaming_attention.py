@@ -197,6 +197,19 @@ def qk_rmsnorm(x: np.ndarray, weight: np.ndarray, eps: float) -> np.ndarray:
     return x / np.sqrt(ms + float(eps)) * w
 
 
+def linear(x: np.ndarray, weight: np.ndarray, round_out: bool = False) -> np.ndarray:
+    """Projection ``y = x W^T`` of the attention block around the path (Q, K, V and output
+    projections of the Qwen3 backbones; not part of the paper's method): ``x [T, K]``,
+    ``weight [N, K]`` (one row per output feature), fp64. ``round_out`` rounds the result to
+    bf16, which is what feeds the attention calls (their q/k/v are bf16)."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64)
+    if x.ndim != 2 or w.ndim != 2 or x.shape[1] != w.shape[1]:
+        raise ValueError("x [T, K] and weight [N, K] are required")
+    y = x @ w.T
+    return round_to_bf16(y) if round_out else y
+
+
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Nearest bf16 value (ties to even) of each fp64 element, returned as fp64.
 

@@ -306,6 +306,32 @@ def test_qk_rmsnorm_pins():
     assert np.array_equal(np.concatenate([ks, kr]), want_k)
 
 
+def test_linear_pins():
+    """The projection against a triple loop, against an identity and a selection matrix, and its bf16 rounding
+    against torch's conversion."""
+    rng = np.random.default_rng(41)
+    T, K, N = 5, 7, 4
+    x, w = rng.standard_normal((T, K)), rng.standard_normal((N, K))
+    want = np.zeros((T, N))
+    for t in range(T):
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                acc += float(x[t, k]) * float(w[n, k])
+            want[t, n] = acc
+    got = osa.linear(x, w)
+    assert np.abs(got - want).max() < 1e-13
+    assert np.array_equal(osa.linear(x, np.eye(K)), x)
+    sel = np.zeros((2, K)); sel[0, 3] = 1.0; sel[1, 0] = -2.0
+    assert np.array_equal(osa.linear(x, sel), np.stack([x[:, 3], -2.0 * x[:, 0]], axis=1))
+    rounded = osa.linear(x, w, round_out=True)
+    via_torch = torch.from_numpy(want).to(torch.float32).to(torch.bfloat16).double().numpy()
+    assert np.abs(rounded - via_torch).max() <= np.abs(want).max() * 2.0 ** -8   # (torch rounds fp32, a double rounding)
+    assert (rounded == via_torch).mean() > 0.9 and np.abs(rounded - want).max() <= np.abs(want).max() * 2.0 ** -8
+    with pytest.raises(ValueError):
+        osa.linear(x, w.T)
+
+
 def test_softmax_rows():
     rng = np.random.default_rng(7)
     n, m, f = [3, 4, 2], [2, 3, 1], 3
