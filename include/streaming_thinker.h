@@ -345,6 +345,27 @@ ST_API int st_decode_attention_static(int32_t device, const void *pool_source, i
  * ST_ERR_CUDA. Like the call it reports on, it allocates nothing; the paper has no counterpart. */
 ST_API int st_decode_static_status(int32_t device, void *stream);
 
+/* Projection y = x W^T on the tensor cores: the Q, K, V and output projections of the attention block around the
+ * path (the Qwen3 backbones of Section 4.1; the paper's method starts behind them, so there is no passage to cite).
+ * x: device bf16 [m, k] row-major with leading dimension ldx (elements); w: device bf16 [n, k] row-major, one row per
+ * output feature (leading dimension ldw); y: device [m, n] row-major (leading dimension ldy), bf16 or, with
+ * out_fp32 != 0, fp32; fp32 accumulation. k and n must be multiples of 8, all three base pointers 16-byte aligned
+ * and every leading dimension a multiple of 16 bytes. The caller owns all buffers; the call is asynchronous on
+ * `stream`. Needs no st_ctx. The first call on a device allocates a 4-byte status word and sets kernel attributes
+ * (make it outside stream capture). err / err_cap: optional HOST buffer for a message. The call makes `device`
+ * current while it runs and restores the caller's device. */
+ST_API int st_linear(int32_t device, const void *x, int64_t m, int64_t k, int64_t ldx, const void *w, int64_t n, int64_t ldw,
+                     void *y, int64_t ldy, int32_t out_fp32, void *stream, char *err, int32_t err_cap);
+
+/* Waits for `stream` and returns ST_OK, or ST_ERR_DEVICE_TIMEOUT if a bounded wait inside an st_linear kernel ran out
+ * since the last call of this function (which clears the word); ST_ERR_INVALID_ARG before the first st_linear on the
+ * device. */
+ST_API int st_linear_status(int32_t device, void *stream);
+
+/* fp32 -> bf16 (round to nearest even) of n contiguous values (n a multiple of 8, both pointers 16-byte aligned,
+ * device memory): turns attention rows into the operand of the output projection. Asynchronous on `stream`. */
+ST_API int st_cast_to_bf16(int32_t device, const void *src, void *dst, int64_t n, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -76,6 +76,10 @@ _SIGS = {
                                              _i32p, _i32p, _i32p, C.c_int32, _vp, _vp, C.c_int32, C.c_int32, C.c_float,
                                              _vp, C.c_char_p, C.c_int32]),
     "st_decode_static_status": (C.c_int, [C.c_int32, _vp]),
+    "st_linear": (C.c_int, [C.c_int32, _vp, C.c_int64, C.c_int64, C.c_int64, _vp, C.c_int64, C.c_int64, _vp, C.c_int64,
+                            C.c_int32, _vp, C.c_char_p, C.c_int32]),
+    "st_linear_status": (C.c_int, [C.c_int32, _vp]),
+    "st_cast_to_bf16": (C.c_int, [C.c_int32, _vp, _vp, C.c_int64, _vp]),
 }
 EXPORTED = tuple(_SIGS)
 for _name, (_res, _args) in _SIGS.items():
@@ -316,3 +320,20 @@ def decode_attention_static(device, pool_source, n_pages_source, pool_reason, n_
 def decode_static_status(device, stream=None) -> int:
     """st_decode_static_status: status code of the most recent allocation-free decode call on the device."""
     return int(lib.st_decode_static_status(device, _ptr(stream)))
+
+
+def linear(device, x, m, k, ldx, w, n, ldw, y, ldy, out_fp32=False, stream=None, check=True):
+    """st_linear: y[m, n] = x[m, k] w[n, k]^T on the tensor cores (pointers: torch tensors, arrays or addresses)."""
+    err = C.create_string_buffer(256)
+    rc = lib.st_linear(device, _ptr(x), m, k, ldx, _ptr(w), n, ldw, _ptr(y), ldy, 1 if out_fp32 else 0, _ptr(stream), err, 256)
+    if rc != ST_OK and check:
+        raise StError(rc, err.value.decode())
+    return rc, err.value.decode()
+
+
+def linear_status(device, stream=None) -> int:
+    return int(lib.st_linear_status(device, _ptr(stream)))
+
+
+def cast_to_bf16(device, src, dst, n, stream=None) -> int:
+    return int(lib.st_cast_to_bf16(device, _ptr(src), _ptr(dst), n, _ptr(stream)))

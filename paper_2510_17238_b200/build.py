@@ -14,7 +14,8 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG_DIR), "include")
 LIB_PATH = os.path.join(PKG_DIR, "libstreaming_thinker.so")
-SOURCES = ["st_api.cu", "st_cache.cu", "st_attn_ref.cu", "st_decode.cu", "st_decode_static.cu", "st_attn_tc.cu"]
+SOURCES = ["st_api.cu", "st_cache.cu", "st_attn_ref.cu", "st_decode.cu", "st_decode_static.cu", "st_attn_tc.cu",
+           "st_linear.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

@@ -46,6 +46,7 @@ constexpr int kDevOk = 0;
 constexpr int kDevTimeoutDecode = 1;
 constexpr int kDevTimeoutPrefill = 2;
 constexpr int kDevTimeoutProbe = 3;     // the wait-expiry test kernel
+constexpr int kDevTimeoutLinear = 5;    // the projection kernel
 constexpr int kDevBadPage = 4;          // a page id read from a page table lies outside its pool: the access was skipped
 
 // ------------------------------------------------------------------------------------------
