@@ -63,6 +63,8 @@ def parse_args():
     ap.add_argument("--arrival", action="store_true",
                     help="side measurement: batch / interleaved / streaming routes under the paper's input arrival "
                          "process (150 words per minute); prints its own JSON line")
+    ap.add_argument("--linear", action="store_true",
+                    help="side measurement: the projection kernel on the attention-block shapes; prints its own JSON line")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the compact measurements of workloads 4 and 3 that the default run appends as per_config")
@@ -320,6 +322,45 @@ def run_arrival(args, local_rank):
         "routes": routes, "data": "synthetic",
         "note": "paper, Table 2 (GSM-Symbolic, Qwen3-4B): tokens before reasoning 94.74 (batch) -> 20.77 (streaming); "
                 "Table 4: first-token latency 28.0 s -> 6.2 s; other hardware, context only"}))
+
+
+def run_linear(args, local_rank):
+    """Side measurement (--linear): the projection kernel st_linear on the shapes of the Qwen3-4B attention block of
+    workload 2's appends (4096 tokens per call, hidden 2560, 32 q / 8 kv heads of 128): Q, K/V and output projection,
+    against the measured bf16 burst peak; torch.matmul (cuBLAS) timed beside it for context."""
+    from paper_2510_17238_b200 import api
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream().cuda_stream
+    peaks = measured_peaks()
+    rows = []
+    for name, m, n, k in (("q_proj", 4096, 4096, 2560), ("kv_proj", 4096, 1024, 2560), ("o_proj", 4096, 2560, 4096)):
+        x = torch.randn((m, k), device=dev).to(torch.bfloat16)
+        w = (torch.randn((n, k), device=dev) / k ** 0.5).to(torch.bfloat16)
+        y = torch.empty((m, n), dtype=torch.bfloat16, device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # larger than L2, written between repeats
+
+        def timed(fn, reps=max(3, args.steps * 5)):
+            for _ in range(max(3, args.warmup)):
+                fn()
+            total = 0.0
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(reps):
+                flush.zero_()
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                total += e0.elapsed_time(e1)
+            return total / reps
+        ms = timed(lambda: api.linear(local_rank, x, m, k, k, w, n, k, y, n, stream=stream))
+        ms_lib = timed(lambda: torch.matmul(x, w.t()))
+        assert api.linear_status(local_rank, stream) == api.ST_OK
+        fl = 2.0 * m * n * k
+        rows.append({"shape": name, "m": m, "n": n, "k": k, "us": ms * 1e3, "achieved": fl / ms / 1e9, "unit": "TFLOP/s",
+                     "peak": peaks["bf16_tflops"], "frac": fl / ms / 1e9 / peaks["bf16_tflops"], "of": peaks["source"],
+                     "cublas_us": ms_lib * 1e3, "cublas_tflops": fl / ms_lib / 1e9})
+    print(json.dumps({"metric": "projection kernel st_linear, Qwen3-4B attention-block shapes at 4096 tokens per call",
+                      "dtype": "bf16", "data": "synthetic", "l2": "256 MB written between repeats", "rows": rows}))
 
 
 def oracle_sample(index, scheds, w, rows_per_sample, seed=0):
@@ -592,6 +633,10 @@ def main():
     if args.arrival:
         if rank == 0:
             run_arrival(args, local_rank)
+        return
+    if args.linear:
+        if rank == 0:
+            run_linear(args, local_rank)
         return
 
     plan = runner.make_plan(scheds, mode="decode", lookahead=1)

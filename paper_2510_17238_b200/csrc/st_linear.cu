@@ -6,10 +6,12 @@
 //   W [N, K] bf16, row-major (leading dimension ldw)                one row per output feature
 //   y [M, N] bf16 or fp32, row-major (leading dimension ldy)        fp32 accumulation
 //
-// Shape of the kernel. One CTA computes one 128 x 256 tile of y. Both operands are K-major, so a tile of either is a
+// Shape of the kernel. One CTA per SM walks the 128 x 256 tiles of y (tile index = CTA index + i * grid size); the
+// accumulator is double-buffered in tensor memory (2 x 256 columns), so the epilogue of one tile runs under the MMAs of
+// the next, and the operand ring keeps filling across tile boundaries. Both operands are K-major, so a tile of either is a
 // box of a 2-D tensor map: 64 elements of K (128 bytes, one swizzle atom) by 128 (x) or 256 (W) rows, landed by TMA in
 // the 128-byte-swizzled layout that the MMA's shared-memory descriptors name; rows and K positions past the end of a
-// matrix arrive as zeros. Four stages of 48 KiB. Warp 0 lane 0 issues the TMA loads, warp 1 allocates 256 columns of
+// matrix arrive as zeros. Four stages of 48 KiB. Warp 0 lane 0 issues the TMA loads, warp 1 allocates the 512 columns of
 // tensor memory and issues, per K block, four MMAs of 128 x 256 x 16 (an elected lane; the loop runs warp-uniform),
 // warps 2-5 read the accumulator (one thread per row, 32 columns at a time), convert and store: 64 or 128 contiguous
 // bytes per thread and step. No TMA load carries a cluster multicast. Every mbarrier wait is bounded.
@@ -37,7 +39,8 @@ constexpr int kLinSmem = kStages * (kStageA + kStageB) + 256;
 struct LinBarriers {
   uint64_t full[kStages];
   uint64_t empty[kStages];
-  uint64_t acc_full;
+  uint64_t acc_full[2];    // the MMAs of a tile into accumulator buffer b are complete
+  uint64_t acc_empty[2];   // the four epilogue warps have read buffer b
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -47,7 +50,7 @@ struct LinParams {
   int32_t *status;
   int64_t M, N, K, ldy;
   int32_t out_fp32;
-  int32_t tiles_n;
+  int32_t tiles_n, tiles;
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
@@ -120,7 +123,6 @@ st_k_linear(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
   LinBarriers &bar = *reinterpret_cast<LinBarriers *>(smem + kStages * (kStageA + kStageB));
   volatile int *abort_flag = &bar.abort_flag;
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  const int tile_m = (int)blockIdx.x / p.tiles_n, tile_n = (int)blockIdx.x % p.tiles_n;
   const int k_blocks = (int)((p.K + kBK - 1) / kBK);
 
   if (threadIdx.x == 0) {
@@ -128,12 +130,15 @@ st_k_linear(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
       mbar_init(smem_u32(&bar.full[i]), 1);
       mbar_init(smem_u32(&bar.empty[i]), 1);
     }
-    mbar_init(smem_u32(&bar.acc_full), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bar.acc_full[i]), 1);
+      mbar_init(smem_u32(&bar.acc_empty[i]), 4);
+    }
     bar.abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
-    lin_tmem_alloc(smem_u32(&bar.tmem_base), kBN);
+    lin_tmem_alloc(smem_u32(&bar.tmem_base), 2 * kBN);
     lin_tmem_relinquish();
   }
   grid_dep_launch();
@@ -146,46 +151,71 @@ st_k_linear(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      for (int kb = 0; kb < k_blocks; ++kb) {
-        const int st = kb % kStages;
-        if (!mbar_wait(smem_u32(&bar.empty[st]), ((uint32_t)(kb / kStages) & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutLinear)) break;
-        const uint32_t full = smem_u32(&bar.full[st]);
-        mbar_arrive_expect_tx(full, kStageA + kStageB);
-        tma_load_2d(smem_u32(smem + st * (kStageA + kStageB)), &map_x, kb * kBK, tile_m * kBM, full);
-        tma_load_2d(smem_u32(smem + st * (kStageA + kStageB) + kStageA), &map_w, kb * kBK, tile_n * kBN, full);
+      int it = 0;                                          // K blocks loaded so far, over all tiles of this CTA
+      for (int tile = (int)blockIdx.x; tile < p.tiles; tile += (int)gridDim.x) {
+        const int tile_m = tile / p.tiles_n, tile_n = tile % p.tiles_n;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const int st = it % kStages;
+          ok = mbar_wait(smem_u32(&bar.empty[st]), ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutLinear);
+          if (!ok) break;
+          const uint32_t full = smem_u32(&bar.full[st]);
+          mbar_arrive_expect_tx(full, kStageA + kStageB);
+          tma_load_2d(smem_u32(smem + st * (kStageA + kStageB)), &map_x, kb * kBK, tile_m * kBM, full);
+          tma_load_2d(smem_u32(smem + st * (kStageA + kStageB) + kStageA), &map_w, kb * kBK, tile_n * kBN, full);
+        }
+        if (!ok) break;
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     const uint32_t issue = lin_elect_one();
     bool ok = true;
-    for (int kb = 0; kb < k_blocks && ok; ++kb) {
-      const int st = kb % kStages;
-      ok = mbar_wait(smem_u32(&bar.full[st]), (uint32_t)(kb / kStages) & 1u, abort_flag, p.status, kDevTimeoutLinear);
+    int it = 0, n_tile = 0;
+    for (int tile = (int)blockIdx.x; tile < p.tiles && ok; tile += (int)gridDim.x, ++n_tile) {
+      const int buf = n_tile & 1;
+      // the epilogue must have read what the tile before last left in this buffer
+      ok = mbar_wait(smem_u32(&bar.acc_empty[buf]), ((uint32_t)(n_tile >> 1) & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutLinear);
       if (!ok) break;
       lin_fence_after();
-      const uint64_t ad = lin_desc(smem_u32(smem + st * (kStageA + kStageB)));
-      const uint64_t bd = lin_desc(smem_u32(smem + st * (kStageA + kStageB) + kStageA));
+      const uint32_t d = tmem + (uint32_t)(buf * kBN);
+      for (int kb = 0; kb < k_blocks && ok; ++kb, ++it) {
+        const int st = it % kStages;
+        ok = mbar_wait(smem_u32(&bar.full[st]), (uint32_t)(it / kStages) & 1u, abort_flag, p.status, kDevTimeoutLinear);
+        if (!ok) break;
+        lin_fence_after();
+        const uint64_t ad = lin_desc(smem_u32(smem + st * (kStageA + kStageB)));
+        const uint64_t bd = lin_desc(smem_u32(smem + st * (kStageA + kStageB) + kStageA));
 #pragma unroll
-      for (int ks = 0; ks < kBK / 16; ++ks)
-        lin_mma_ss(tmem, ad + (uint64_t)((ks * 32) >> 4), bd + (uint64_t)((ks * 32) >> 4), kLinIdesc, (kb > 0 || ks > 0) ? 1u : 0u, issue);
-      lin_commit(smem_u32(&bar.empty[st]), issue);      // the stage is free once these MMAs have read it
+        for (int ks = 0; ks < kBK / 16; ++ks)
+          lin_mma_ss(d, ad + (uint64_t)((ks * 32) >> 4), bd + (uint64_t)((ks * 32) >> 4), kLinIdesc, (kb > 0 || ks > 0) ? 1u : 0u, issue);
+        lin_commit(smem_u32(&bar.empty[st]), issue);      // the stage is free once these MMAs have read it
+      }
+      if (ok) lin_commit(smem_u32(&bar.acc_full[buf]), issue);
     }
-    if (ok) lin_commit(smem_u32(&bar.acc_full), issue);
   } else {
     // ------------------------------------------------------------------ epilogue: thread = row = TMEM lane
     const int quarter = warp & 3;                        // the TMEM lanes a warp may read: 32 * (warp % 4) ...
     const int r_local = quarter * 32 + lane;
-    const int64_t row = (int64_t)tile_m * kBM + r_local;
-    const bool ok = mbar_wait(smem_u32(&bar.acc_full), 0, abort_flag, p.status, kDevTimeoutLinear);
-    lin_fence_after();
-    if (ok) {
-      const uint32_t t_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    int n_tile = 0;
+    for (int tile = (int)blockIdx.x; tile < p.tiles; tile += (int)gridDim.x, ++n_tile) {
+      const int tile_m = tile / p.tiles_n, tile_n = tile % p.tiles_n;
+      const int buf = n_tile & 1;
+      const int64_t row = (int64_t)tile_m * kBM + r_local;
+      if (!mbar_wait(smem_u32(&bar.acc_full[buf]), (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kDevTimeoutLinear)) break;
+      lin_fence_after();
+      const uint32_t t_addr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kBN);
 #pragma unroll 1
       for (int c0 = 0; c0 < kBN; c0 += 32) {
         float acc[32];
         lin_tmem_ld32(t_addr + c0, acc);
         lin_wait_ld();
+        if (c0 == kBN - 32) {
+          // the last columns are in registers: the buffer may take the tile after next
+          lin_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bar.acc_empty[buf]));
+        }
         const int64_t col = (int64_t)tile_n * kBN + c0;
         if (row < p.M && col < p.N) {
           // N is a multiple of 8: a group of 8 columns is inside the matrix or outside it
@@ -211,7 +241,7 @@ st_k_linear(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
   __syncthreads();
   if (warp == 1) {
     lin_fence_after();
-    lin_tmem_dealloc(tmem, kBN);
+    lin_tmem_dealloc(tmem, 2 * kBN);
   }
 }
 
@@ -224,6 +254,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 struct LinearDevice {
   bool ready = false;
   int32_t *status = nullptr;
+  int num_sms = 0;
 };
 constexpr int kLinMaxDevices = 64;
 LinearDevice g_lin_device[kLinMaxDevices];
@@ -289,6 +320,7 @@ extern "C" int st_linear(int32_t device, const void *x, int64_t m, int64_t k, in
     LinearDevice &d = g_lin_device[device];
     if (!d.ready) {
       e = cudaFuncSetAttribute(st_k_linear, cudaFuncAttributeMaxDynamicSharedMemorySize, kLinSmem + 1024);
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, device);
       if (e == cudaSuccess) e = cudaMalloc(&d.status, sizeof(int32_t));
       if (e == cudaSuccess) e = cudaMemset(d.status, 0, sizeof(int32_t));
       if (e != cudaSuccess) return lin_fail(err, err_cap, ST_ERR_CUDA, std::string("kernel set-up: ") + cudaGetErrorString(e));
@@ -310,8 +342,9 @@ extern "C" int st_linear(int32_t device, const void *x, int64_t m, int64_t k, in
   p.tiles_n = (int32_t)((n + kBN - 1) / kBN);
   const int64_t tiles = ((m + kBM - 1) / kBM) * p.tiles_n;
   if (tiles > INT32_MAX) return lin_fail(err, err_cap, ST_ERR_INVALID_ARG, "too many output tiles");
+  p.tiles = (int32_t)tiles;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)tiles);
+  cfg.gridDim = dim3((unsigned)std::min<int64_t>(tiles, dev.num_sms));
   cfg.blockDim = dim3(kLinThreads);
   cfg.dynamicSmemBytes = kLinSmem + 1024;
   cfg.stream = (cudaStream_t)stream;
