@@ -355,3 +355,11 @@ def test_packed_forward_positions_visibility_and_state():
     assert ctx.pages_free() == (2, 8)
     ctx = host_ctx(n_pages_source=16, n_pages_reason=8, max_tokens_per_call=total, position_mode=api.ST_POS_UNIT_ALIGNED)
     assert ctx.forward_packed(0, [0], scheds[:1], None, None, None, None, check=False) == api.ST_ERR_INVALID_ARG
+
+
+def test_linear_rejects_bad_arguments():
+    E = api.ST_ERR_INVALID_ARG
+    ok = dict(device=0, x=1024, m=8, k=64, ldx=64, w=2048, n=16, ldw=64, y=4096, ldy=16, check=False)
+    for bad in (dict(k=60), dict(n=12), dict(ldx=56), dict(ldw=68), dict(ldy=8), dict(x=1028), dict(m=0), dict(x=None)):
+        assert api.linear(**{**ok, **bad})[0] == E
+    assert api.cast_to_bf16(0, 1024, 2048, 12) == E
