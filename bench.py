@@ -36,11 +36,11 @@ import numpy as np
 import torch
 
 # DRAM bytes per algorithmic byte of st_k_decode, from an ncu capture of the small decode case (--profile-case decode:
-# 272.8 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
-DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.0177
-# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill); None until the counters of the
-# kernel as it stands have been taken.
-PREFILL_DRAM_PER_ALGORITHMIC_BYTE = None
+# 273.7 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
+DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.019
+# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 147.1 and 158.4 MB moved for 167.8
+# and 176.2 MB of K/V, queries and output rows; below 1 because the rows a launch writes are still in L2 when it ends).
+PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.888
 
 METRIC = "reasoning-decode tok/s per layer (chunk prefill concurrent on a second stream)"
 UNIT = "tok/s"
