@@ -517,7 +517,12 @@ def measure_side_config(index, args, local_rank, layers=None):
                        "peak": peaks["bf16_tflops"], "frac": tflops / peaks["bf16_tflops"], "launches_per_pass": n_pre // 2,
                        "kernel_ms_per_pass": ms_pre, "append_chain_ms_per_pass": ms_chain,
                        "append_chain_tflops": flops / (ms_chain / 1e3) / 1e12,
-                       "prefill_tok_s_chain": sum(s.S for s in scheds) * L / (ms_chain / 1e3)},
+                       "prefill_tok_s_chain": sum(s.S for s in scheds) * L / (ms_chain / 1e3),
+                       # short units make chunk prefill memory-bound (G x tokens per unit below the ridge of ~250 flop/byte):
+                       # the same launches against the copy bandwidth
+                       "algorithmic_GBps": prefill_algorithmic_bytes(scheds, w) * L / (ms_pre / 1e3) / 1e9 if ms_pre > 0 else 0.0,
+                       "frac_of_hbm": (prefill_algorithmic_bytes(scheds, w) * L / (ms_pre / 1e3) / 1e9 / peaks["hbm_gbs"]) if ms_pre > 0 else 0.0,
+                       "mean_packed_rows_per_unit": float(np.mean([n * (w.n_q_heads // w.n_kv_heads) for s in scheds for n in s.src_unit_len]))},
            "of": peaks["source"], "clocks": clocks}
     ctx.close()
     del batch, compiled
