@@ -76,6 +76,11 @@ struct st_ctx {
   double2 *rope_hi = nullptr, *rope_lo = nullptr;   // rotation tables of the fused decode append
   float *d_norm = nullptr;                          // q/k normalisation weights [layer][q, k][128], or nullptr
   int32_t *d_status = nullptr;
+  // key-split workspace of the tensor-core attention kernel, per side (source appends and reasoning spans may run on
+  // two streams at once): un-normalised outputs, (maximum, row sum) pairs, tickets
+  float *split_o[2] = {nullptr, nullptr};
+  float2 *split_ml[2] = {nullptr, nullptr};
+  int32_t *split_ticket[2] = {nullptr, nullptr};
   // staging for ST_IO_HOST, per side
   __nv_bfloat16 *stage_q[2] = {nullptr, nullptr}, *stage_k[2] = {nullptr, nullptr}, *stage_v[2] = {nullptr, nullptr};
   float *stage_out[2] = {nullptr, nullptr};
@@ -169,6 +174,9 @@ void release_device(st_ctx *ctx) {
     cudaFree(ctx->stage_k[s]);
     cudaFree(ctx->stage_v[s]);
     cudaFree(ctx->stage_out[s]);
+    cudaFree(ctx->split_o[s]);
+    cudaFree(ctx->split_ml[s]);
+    cudaFree(ctx->split_ticket[s]);
   }
   cudaFree(ctx->partial);
   cudaFree(ctx->rope_hi);
@@ -517,6 +525,10 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
   p->norm_k = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 + 128 : nullptr;
   p->norm_eps = ctx->cfg.qk_norm_eps;
   p->total_work = p->work_per_cta = p->n_cta = 0;
+  p->split_o = ctx->split_o[side];
+  p->split_ml = ctx->split_ml[side];
+  p->split_ticket = ctx->split_ticket[side];
+  p->n_split = 0;
 }
 
 // Attention for the rows of a call. kind: 0 chunk prefill, 1 decode, 2 extend.
@@ -524,9 +536,17 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
 // Launches the attention kernels of one call for a list of work entries (one per sequence for the streaming calls,
 // one per (sequence, reasoning unit) for the packed forward). kind: 0 chunk prefill, 1 decode, 2 spans.
 // `fused`: a decode step whose append runs inside the decode kernel (the call's un-rotated q/k/v).
-int launch_attention_entries(st_ctx *ctx, int kind, int32_t layer, const std::vector<st::AttnSeq> &entries, int total_rows,
+int launch_attention_entries(st_ctx *ctx, int kind, int32_t layer, const std::vector<st::AttnSeq> &entries_in, int total_rows,
                              float *out, uint32_t flags, cudaStream_t stream, const IoPtrs &io, bool fused) {
   const int side = kind == 0 ? 0 : 1;
+  // The tensor-core kernel's CTAs are handed out in entry order and an entry's CTAs all walk about the same number of
+  // keys: longest entries first, so that the last, partly filled wave of a ragged call holds the short ones (the
+  // decode kernel cuts its tile list into equal slices and needs no such order).
+  std::vector<st::AttnSeq> entries(entries_in);
+  if (kind != 1)
+    std::stable_sort(entries.begin(), entries.end(), [](const st::AttnSeq &a, const st::AttnSeq &b) {
+      return (int64_t)a.a_len + a.b_base + a.n_rows > (int64_t)b.a_len + b.b_base + b.n_rows;
+    });
   for (size_t s0 = 0; s0 < entries.size(); s0 += st::kMaxSeqPerLaunch) {
     const int ns = (int)std::min<size_t>(st::kMaxSeqPerLaunch, entries.size() - s0);
     st::AttnParams ap;
@@ -994,6 +1014,13 @@ int st_create(const st_config *cfg, st_ctx **out) {
     ctx->cfg.q_norm_weight = ctx->cfg.k_norm_weight = nullptr;   // (the caller's arrays are not used after this call)
     ST_CREATE_CUDA(cudaMalloc(&ctx->d_status, sizeof(int32_t)));
     ST_CREATE_CUDA(cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    for (int s = 0; s < 2; ++s) {
+      const size_t rows = (size_t)st::kMaxSplitItems * 2 * st::attn_tc_rows_per_cta();
+      ST_CREATE_CUDA(cudaMalloc(&ctx->split_o[s], rows * st::kHeadDim * sizeof(float)));
+      ST_CREATE_CUDA(cudaMalloc(&ctx->split_ml[s], rows * sizeof(float2)));
+      ST_CREATE_CUDA(cudaMalloc(&ctx->split_ticket[s], st::kMaxSplitItems * 2 * sizeof(int32_t)));
+      ST_CREATE_CUDA(cudaMemset(ctx->split_ticket[s], 0, st::kMaxSplitItems * 2 * sizeof(int32_t)));
+    }
     ST_CREATE_CUDA(cudaDeviceSynchronize());
   }
 #undef ST_CREATE_CUDA
@@ -1195,6 +1222,8 @@ int st_device_status(st_ctx *ctx) {
   ST_CUDA(ctx, cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
   if (h != st::kDevOk) {
     ST_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    // (a kernel that gave up may have left a key-split ticket odd)
+    for (int s = 0; s < 2; ++s) ST_CUDA(ctx, cudaMemset(ctx->split_ticket[s], 0, st::kMaxSplitItems * 2 * sizeof(int32_t)));
     if (h == st::kDevBadPage)
       return fail(ctx, ST_ERR_DEVICE_CHECK, "a page id read from a page table lies outside its pool; the access was skipped");
     return fail(ctx, ST_ERR_DEVICE_TIMEOUT, h == st::kDevTimeoutDecode    ? "a bounded wait expired in the decode kernel"

@@ -41,6 +41,7 @@
 // range and leaves the result exact (the same reference is used for P, l and O). The row sum adds the
 // bf16-rounded probabilities, i.e. exactly the weights the tensor core applies to V.
 // Every mbarrier wait is bounded; on expiry the CTA records a status word, stops and frees its TMEM.
+#include <algorithm>
 #include <cstddef>
 
 #include "st_internal.h"
@@ -61,6 +62,8 @@ constexpr int kKStageBytes = 32768;         // 2 channel halves x 128 keys x 128
 constexpr int kVStageBytes = 32768;         // 2 pages x 128 channels x 128 B (64 keys)
 constexpr int kHalfPanel = 16384;           // one channel half of a 128-row tile / one V^T page panel
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr int kMinCutPages = 20;             // key split: items of fewer cache pages are not cut (below about ten key
+                                            // tiles the merge costs more than the shorter last wave saves)
 #ifndef ST_ATTN_POLY_PAIRS
 #define ST_ATTN_POLY_PAIRS 0x92u
 #endif
@@ -288,26 +291,51 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
   const uint32_t g_magic = (uint32_t)((0x100000000ull + (uint32_t)G - 1u) / (uint32_t)G);
   auto div_g = [&](int row) { return G == 1 ? row : (int)__umulhi((uint32_t)row, g_magic); };
 
-  // ---- which (sequence, kv head, row pair) is this CTA
-  const int s = last_not_above(p.n_seq, (int)blockIdx.x, [&](int i) { return p.seq[i].work_begin; });
+  // ---- which work item (sequence, kv head, row pair) is this CTA, and which part of its keys.
+  // The last n_split items of the launch are run by two CTAs each (CTA indices from first_split on, two per item).
+  const int first_split = p.total_work - p.n_split;
+  int item = (int)blockIdx.x, part = -1;                     // part -1: all keys of the item
+  if (item >= first_split) {
+    const int k = item - first_split;
+    item = first_split + (k >> 1);
+    part = k & 1;
+  }
+  const int split_idx = item - first_split;
+  const int s = last_not_above(p.n_seq, item, [&](int i) { return p.seq[i].work_begin; });
   const AttnSeq sq = p.seq[s];
   const int packed_rows = sq.n_rows * G;
   const int pairs = (packed_rows + kRowsPerCta - 1) / kRowsPerCta;
-  const int rel = (int)blockIdx.x - sq.work_begin;
+  const int rel = item - sq.work_begin;
   const int kvh = rel / pairs, pair = rel - kvh * pairs;
   const int row0 = pair * kRowsPerCta;                       // first packed row of the CTA
 
   // per M-tile geometry: pages (range A pages, then range B pages) and 128-key tiles
   const int nA = (sq.a_len + 63) >> 6;
+  int np_all[2], n_pages_all = 0;                            // pages each M-tile looks at, over all keys of the item
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r_lo = row0 + t * kRowsPerTile;
+    const int r_hi = min(r_lo + kRowsPerTile, packed_rows) - 1;
+    np_all[t] = r_lo < packed_rows ? nA + ((sq.b_base + r_hi / G) >> 6) + 1 : 0;
+    n_pages_all = max(n_pages_all, np_all[t]);
+  }
+  // Key split. An item of at least kMinCutPages pages is cut at a tile boundary near its middle: part 0 takes the pages in
+  // front of page_mid, part 1 those from page_mid on (M-tile 0 looks at no less than the item's page count minus two,
+  // so both parts of both M-tiles are non-empty). Each part leaves un-normalised outputs with its reference maxima and
+  // row sums in the workspace; whichever part of an M-tile finishes second adds the two and writes the rows out. A
+  // shorter item is not cut: part 0 does all of it, part 1 has nothing to do.
+  const bool cut = part >= 0 && n_pages_all >= kMinCutPages;
+  const int page_mid = 2 * (((n_pages_all + 1) >> 1) >> 1);
+  const int pg0 = cut && part == 1 ? page_mid : 0;           // first page of this CTA's share
   int n_tiles[2];
   bool active[2];
   int n_pages = 0;
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
-    const int r_lo = row0 + t * kRowsPerTile;
-    active[t] = r_lo < packed_rows;
-    const int r_hi = min(r_lo + kRowsPerTile, packed_rows) - 1;
-    const int np = active[t] ? nA + ((sq.b_base + r_hi / G) >> 6) + 1 : 0;
+    int np = np_all[t];
+    if (cut) np = part == 0 ? min(np, page_mid) : max(np - page_mid, 0);
+    if (!cut && part == 1) np = 0;
+    active[t] = np > 0;
     n_tiles[t] = (np + 1) >> 1;
     n_pages = max(n_pages, np);
   }
@@ -505,7 +533,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           }
 
           // visible columns of this row in this page: column c is visible iff c <= lim
-          const int pg = 2 * j + h;
+          const int pg = pg0 + 2 * j + h;
           const int lim = pg < nA ? sq.a_len - (pg << 6) - 1 : sq.b_base + tok - ((pg - nA) << 6);
           if (lim < 63) {
 #pragma unroll
@@ -610,33 +638,91 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       // passes whatever happened before, so the group barrier cannot be left waiting.
       const bool fin = ok && mbar_wait(smem_u32(&bar.o_final[t]), 0, abort_flag, p.status, kDevTimeoutPrefill);
       tc_fence_after();
-      const float inv = 1.f / l_sum;
       uint8_t *stage = smem + kOffQ + t * kQTileBytes;        // 128 rows x 256 bytes
+      // The tile's accumulator to the output rows: this thread's row times `mul`; with `other` set, plus the other
+      // part's share of the row (workspace, in the layout of write_share below) times `other_mul`.
+      auto write_rows = [&](float mul, const float4 *other, float other_mul) {
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float ov[32];
+        for (int half = 0; half < 2; ++half) {
+          float ov[32];
 #pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 32) {
-          tmem_ld32(o_addr + half * 64 + c0, ov);
+          for (int c0 = 0; c0 < 64; c0 += 32) {
+            tmem_ld32(o_addr + half * 64 + c0, ov);
+            float4 o[8];
+            if (other) {
+#pragma unroll
+              for (int c = 0; c < 8; ++c) o[c] = __ldcg(other + (size_t)((half * 64 + c0) / 4 + c) * kRowsPerTile + r_local);
+            }
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+              // (each product is rounded on its own - no fused multiply-add - and the sum commutes: the bits do not
+              // depend on which part merges)
+              float4 v = make_float4(__fmul_rn(ov[c], mul), __fmul_rn(ov[c + 1], mul), __fmul_rn(ov[c + 2], mul), __fmul_rn(ov[c + 3], mul));
+              if (other) {
+                const float4 w = o[c >> 2];
+                v = make_float4(__fadd_rn(v.x, __fmul_rn(w.x, other_mul)), __fadd_rn(v.y, __fmul_rn(w.y, other_mul)),
+                                __fadd_rn(v.z, __fmul_rn(w.z, other_mul)), __fadd_rn(v.w, __fmul_rn(w.w, other_mul)));
+              }
+              *reinterpret_cast<float4 *>(stage + r_local * 256 + ((((c0 + c) >> 2) ^ (r_local & 15)) << 4)) = v;
+            }
+          }
+          tile_sync(t);
+          const int c = r_local & 15;
+#pragma unroll 4
+          for (int i = 0; i < 16; ++i) {
+            const int rr = i * 8 + (r_local >> 4);
+            const int grow = row0 + t * kRowsPerTile + rr;
+            const float4 v = *reinterpret_cast<const float4 *>(stage + rr * 256 + ((c ^ (rr & 15)) << 4));
+            if (fin && grow < packed_rows) {
+              const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
+              *reinterpret_cast<float4 *>(p.out + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + half * 64 + c * 4) = v;
+            }
+          }
+          tile_sync(t);
+        }
+      };
+      // This part's un-normalised share of the tile to the workspace, straight from tensor memory: 16-byte chunk q of
+      // row r at [q][r], so that a warp's 32 rows write (and the merging part reads) 512 contiguous bytes.
+      auto write_share = [&](float4 *share) {
+#pragma unroll
+        for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+          float ov[32];
+          tmem_ld32(o_addr + c0, ov);
           tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < 32; c += 4)
-            *reinterpret_cast<float4 *>(stage + r_local * 256 + ((((c0 + c) >> 2) ^ (r_local & 15)) << 4)) =
-                make_float4(ov[c] * inv, ov[c + 1] * inv, ov[c + 2] * inv, ov[c + 3] * inv);
+            share[(size_t)((c0 + c) >> 2) * kRowsPerTile + r_local] = make_float4(ov[c], ov[c + 1], ov[c + 2], ov[c + 3]);
         }
-        tile_sync(t);
-        const int c = r_local & 15;
-#pragma unroll 4
-        for (int i = 0; i < 16; ++i) {
-          const int rr = i * 8 + (r_local >> 4);
-          const int grow = row0 + t * kRowsPerTile + rr;
-          const float4 v = *reinterpret_cast<const float4 *>(stage + rr * 256 + ((c ^ (rr & 15)) << 4));
-          if (fin && grow < packed_rows) {
-            const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
-            *reinterpret_cast<float4 *>(p.out + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + half * 64 + c * 4) = v;
-          }
+      };
+      if (!cut) {
+        write_rows(1.f / l_sum, nullptr, 0.f);
+      } else {
+        // This part's share goes to the workspace; the ticket of (item, M-tile) then tells whether the other part was
+        // there first (odd count: tickets are never reset, each launch adds two).
+        const size_t mine = (size_t)(split_idx * 2 + part) * kRowsPerCta + t * kRowsPerTile;
+        const size_t theirs = (size_t)(split_idx * 2 + (part ^ 1)) * kRowsPerCta + t * kRowsPerTile;
+        float4 *share = reinterpret_cast<float4 *>(p.split_o);
+        if (fin) {
+          p.split_ml[mine + r_local] = make_float2(m_ref, l_sum);
+          write_share(share + mine * (kHeadDim / 4));
         }
+        __threadfence();
         tile_sync(t);
+        // (all four warps of the tile take the same path from here whatever happened before: the group barriers
+        // cannot be left waiting; a tile that gave up takes no ticket and writes nothing)
+        int *second = reinterpret_cast<int *>(smem + kOffP1 + t * kP1Bytes);   // free: the last P V is complete
+        if (r_local == 0) *second = fin ? atomicAdd(p.split_ticket + split_idx * 2 + t, 1) & 1 : 0;
+        tile_sync(t);
+        if (*second) {
+          __threadfence();
+          const float2 o_ml = __ldcg(p.split_ml + theirs + r_local);
+          // (a part in which this row saw no key has maximum -inf and weight 0; part 0 always sees the first key)
+          const float m_all = fmaxf(m_ref, o_ml.x);
+          const float w_mine = exp2_approx(m_ref - m_all), w_theirs = exp2_approx(o_ml.x - m_all);
+          const float inv = __frcp_rn(__fadd_rn(__fmul_rn(l_sum, w_mine), __fmul_rn(o_ml.y, w_theirs)));
+          write_rows(__fmul_rn(w_mine, inv), share + theirs * (kHeadDim / 4), __fmul_rn(w_theirs, inv));
+        }
       }
       tc_fence_before();
     }
@@ -649,7 +735,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         bool pages_ok = true;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const int pg = min(2 * j + h, n_pages - 1);
+          const int pg = pg0 + min(2 * j + h, n_pages - 1);
           const bool in_a = pg < nA;
           const int page = in_a ? p.ptab_a[(size_t)sq.slot * p.ptab_stride_a + pg]
                                 : p.ptab_b[(size_t)sq.slot * p.ptab_stride_b + (pg - nA)];
@@ -812,7 +898,6 @@ int attn_tc_rows_per_cta() { return kRowsPerCta; }
 
 cudaError_t launch_attn_tc(AttnParams &p, bool precise, int num_sms, cudaStream_t stream, int *n_launches, cudaEvent_t t0,
                            cudaEvent_t t1) {
-  (void)num_sms;
   *n_launches = 0;
   int total = 0;
   for (int i = 0; i < p.n_seq; ++i) {
@@ -821,11 +906,24 @@ cudaError_t launch_attn_tc(AttnParams &p, bool precise, int num_sms, cudaStream_
   }
   if (total == 0) return cudaSuccess;
   p.total_work = total;
-  p.n_cta = total;
+  // One CTA per SM at a time: the items run in waves of num_sms. When the last wave would fill at most half of the
+  // SMs, its items are cut in two by keys (two CTAs each), so that it takes about half as long.
+  const int tail = total % num_sms;
+  p.n_split = (p.split_o != nullptr && tail > 0 && 2 * tail <= num_sms) ? std::min(tail, kMaxSplitItems) : 0;
+  if (p.n_split > 0) {   // ... unless none of them is long enough to be cut (the kernel decides per item, by the same count)
+    int longest = 0;
+    for (int i = p.n_seq - 1; i >= 0; --i) {
+      const AttnSeq &sq = p.seq[i];
+      if (sq.n_rows > 0) longest = std::max(longest, ((sq.a_len + 63) >> 6) + ((sq.b_base + sq.n_rows - 1) >> 6) + 1);
+      if (sq.work_begin <= total - p.n_split) break;
+    }
+    if (longest < kMinCutPages) p.n_split = 0;
+  }
+  p.n_cta = total + p.n_split;
   if (t0) cudaEventRecord(t0, stream);
   // (the two-term variant takes queries that the append kernel has normalised and rotated)
   auto kernel = precise ? st_k_attn_tc<true, false> : p.norm_q != nullptr ? st_k_attn_tc<false, true> : st_k_attn_tc<false, false>;
-  cudaError_t e = launch_dependent(kernel, dim3(total), dim3(kThreads), kSmemBytes + 1024, stream, p);
+  cudaError_t e = launch_dependent(kernel, dim3(p.n_cta), dim3(kThreads), kSmemBytes + 1024, stream, p);
   if (e != cudaSuccess) return e;
   if (t1) cudaEventRecord(t1, stream);
   *n_launches = 1;

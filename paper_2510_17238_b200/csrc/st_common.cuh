@@ -31,6 +31,7 @@ constexpr int kBlockBytes = 32768;
 constexpr int kKeyBytes = 16384;
 constexpr int kPanelBytesK = 8192;
 constexpr int kRopeLoSteps = 1024;      // positions covered by the fine rotation table
+constexpr int kMaxSplitItems = 74;     // work items of one tensor-core attention launch that may be split by keys
 constexpr int kMaxSeqPerLaunch = 112;   // keeps every parameter block under the 4 KiB limit
 constexpr int kMaxGroup = 8;            // q heads per kv head
 
@@ -115,6 +116,13 @@ struct AttnParams {
   float norm_eps;
   // decode with the append fused in: (cos, sin) of k * 1024 * inv_freq[c] and of j * inv_freq[c], j < 1024, as [.][64]
   const double2 *rope_hi, *rope_lo;
+  // Tensor-core kernel, key split of the last work items of a launch (see st_k_attn_tc): the last n_split items are
+  // run by two CTAs each, one per half of the keys; whichever finishes second merges. Workspace per split item and
+  // half: 256 rows x 128 un-normalised outputs, 256 x (reference maximum, row sum); one ticket per item and M-tile.
+  float *split_o;
+  float2 *split_ml;
+  int32_t *split_ticket;
+  int32_t n_split;
   AttnSeq seq[kMaxSeqPerLaunch];
 };
 static_assert(sizeof(AttnParams) <= 4096, "kernel parameter space");
