@@ -38,9 +38,9 @@ import torch
 # DRAM bytes per algorithmic byte of st_k_decode, from an ncu capture of the small decode case (--profile-case decode:
 # 273.7 MB moved for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to capture.
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.019
-# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 147.1 and 158.4 MB moved for 167.8
-# and 176.2 MB of K/V, queries and output rows; below 1 because the rows a launch writes are still in L2 when it ends).
-PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.888
+# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 192.5 and 204.5 MB moved for 209.7
+# and 220.2 MB of K/V, queries and output rows; below 1 because the rows a launch writes are still in L2 when it ends).
+PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.923
 
 METRIC = "reasoning-decode tok/s per layer (chunk prefill concurrent on a second stream)"
 UNIT = "tok/s"
@@ -554,15 +554,17 @@ def run_reference(args, w, scheds, rank, world):
 
 
 def profile_case(kind):
-    """A small case of the same kernels for profiler captures: 16 sequences of config 2's head shape.
+    """A small case of the same kernels for profiler captures: 16 (decode) or 20 (prefill) sequences of config 2's
+    head shape.
 
     decode : 2048 source tokens (one append) + 2040 reasoning tokens (one span) per sequence, then 8 decode
              steps at ~4090 keys per sequence: 268 MB of K/V per step (larger than L2), 8 st_k_decode launches.
     prefill: sixteen 128-token units appended one after the other (prefix 0 .. 1920): 16 st_k_attn_tc launches
-             of 256 CTAs; the last ones are the representative ones."""
+             of 320 work items (two full waves on 148 SMs and 24 items that the kernel cuts in two by keys once they
+             hold 20 pages); the last ones are the representative ones."""
     from paper_2510_17238_b200 import api, workloads
     w = workloads.WORKLOADS[2]
-    B, S, R = 16, 2048, 2048
+    B, S, R = (20 if kind == "prefill" else 16), 2048, 2048
     sched = workloads.SeqSchedule((S,), (R,), 0)
     dev = torch.device("cuda", 0)
     cfg = api.make_config(n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, max_batch=B, n_pages_source=B * S // 64,
@@ -671,6 +673,17 @@ def main():
         torch.cuda.synchronize()
         return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
+    # ---- chunk prefill alone: the same appends with no decode stream beside them, so that the tensor-core
+    # kernel's own rate is seen (in the concurrent pass its launches share the SMs with the decode kernel). It runs
+    # first, a burst on a GPU that has not been under load for seconds, which is how the peak it is compared with
+    # was measured (under the power cap the SM clock settles some 2-4 % lower during the long timed region below).
+    solo_reps = 5
+    solo_sampler = ClockSampler(local_rank)
+    if rank == 0:
+        solo_sampler.start()
+    n_pre_solo, ms_pre_solo, ms_chain = measure_prefill_alone(ctx, compiled, api, solo_reps)
+    solo_clocks = solo_sampler.stop() if rank == 0 else None
+
     for _ in range(args.warmup):
         one_pass(compiled)
     torch.cuda.synchronize()
@@ -689,10 +702,6 @@ def main():
     gpu_launches = ctx.launch_count() - launches0
     ctx.device_status()
 
-    # ---- chunk prefill alone: the same appends with no decode stream beside them, so that the tensor-core
-    # kernel's own rate is seen (in the concurrent pass its launches share the SMs with the decode kernel)
-    solo_reps = 5
-    n_pre_solo, ms_pre_solo, ms_chain = measure_prefill_alone(ctx, compiled, api, solo_reps)
 
     B = len(scheds)
     rsn_tokens = sum(s.R for s in scheds)
@@ -730,7 +739,8 @@ def main():
                         "of": peaks["source"] + " (burst: kernel timed alone, appends only, no decode stream)",
                         "frac_of_sustained": solo_tflops / peaks["bf16_tflops_sustained"],
                         "frac_of_nominal_2250": solo_tflops / 2250.0,
-                        "launches": n_pre_solo, "total_ms_per_pass": ms_pre_solo,
+                        "launches": n_pre_solo, "total_ms_per_pass": ms_pre_solo, "clocks": solo_clocks,
+                        "when": "before the warm-up passes of the timed region",
                         "algorithmic_flops_per_pass": pre_flops,
                         "traffic": PREFILL_DRAM_PER_ALGORITHMIC_BYTE * pre_bytes / max(n_pre_solo // solo_reps, 1)
                         if PREFILL_DRAM_PER_ALGORITHMIC_BYTE else None,

@@ -66,22 +66,30 @@ def test_ragged_edges(hq):
         assert pu.check_cache(ctx, w, scheds, plan, flats[0]) <= 2
 
 
-@pytest.mark.parametrize("hq", [8, 32, 40])
-def test_key_split_of_long_items(hq):
+@pytest.mark.parametrize("hq,variant", [(8, "plain"), (32, "plain"), (40, "plain"), (40, "two_term"), (16, "qk_norm")])
+def test_key_split_of_long_items(hq, variant):
     """Work items of twenty and more cache pages in a launch that fills less than half of the SMs: the tensor-core
     kernel cuts each of them in two by keys and the part that finishes second merges. Twenty pages exactly and
     nineteen (not cut), a source prefix that ends inside a page (odd and even page counts in front of the reasoning
-    pages), a second row pair with an empty second M-tile; group sizes 1, 4 and 5."""
+    pages), a second row pair with an empty second M-tile; group sizes 1, 2, 4 and 5; the one-term, the two-term and
+    the normalising instantiation of the kernel."""
     w = small_workload(hq)
     scheds = [
         workloads.SeqSchedule((1217, 300, 70), (130, 257, 64), 40),     # 19 pages behind the first unit, then more
         workloads.SeqSchedule((1230, 50, 5), (0, 200, 3), 0),           # second unit: last row in page 19 (20 pages)
         workloads.SeqSchedule((1152, 63, 129), (1, 300, 2), 17),        # second unit: 19 pages, third: 21
     ]
-    ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode="extend", lookahead=1)
-    worst = pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], n_random=160, what=f"key split hq={hq}")
-    assert pu.check_cache(ctx, w, scheds, plan, flats[0], seqs=(1,)) <= 2
-    print("key split", hq, "worst (max_abs, rel_l2):", worst)
+    flags = api.ST_CFG_PRECISE_P if variant == "two_term" else 0
+    norm = None
+    if variant == "qk_norm":
+        rng = np.random.default_rng(5)
+        norm = (rng.uniform(0.5, 1.5, size=(1, 128)).astype(np.float32), rng.uniform(0.5, 1.5, size=(1, 128)).astype(np.float32), 1e-6)
+    ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode="extend", lookahead=1, cfg_flags=flags, qk_norm=norm)
+    norm0 = None if norm is None else (norm[0][0], norm[1][0], norm[2])
+    worst = pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], n_random=160, what=f"key split hq={hq} {variant}",
+                                    qk_norm=norm0)
+    assert pu.check_cache(ctx, w, scheds, plan, flats[0], seqs=(1,), k_norm=None if norm is None else (norm[1][0], norm[2])) <= 2
+    print("key split", hq, variant, "worst (max_abs, rel_l2):", worst)
 
 
 def test_ragged_edges_with_sentinel_filled_pages():
