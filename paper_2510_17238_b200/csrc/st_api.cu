@@ -48,6 +48,7 @@ struct Pending {
   std::vector<int32_t> rope_off;      // per listed sequence: position id of a new token minus its index in the cache
   std::vector<uint8_t> is_final;      // per listed sequence: the call named ST_VIS_ALL (final depth)
   uint64_t wait_serial = 0;
+  bool reverse = false;               // decode step: the kernel walks its tile list backwards (see st_k_decode)
 };
 
 thread_local std::string g_create_error;
@@ -108,6 +109,7 @@ struct st_ctx {
   bool precise_p = false;        // ST_CFG_PRECISE_P: two-term probabilities in the tensor-core attention kernel
   bool poison = false;           // ST_CFG_DEBUG_CHECKS: free pages hold a large finite sentinel instead of zeros
   int fail_countdown = 0;        // test hook: the n-th internal device step from now reports ST_ERR_CUDA
+  uint64_t decode_steps = 0;     // decode steps issued since the last full reset: odd ones walk the caches backwards
 };
 
 namespace {
@@ -525,6 +527,7 @@ void fill_attn_common(st_ctx *ctx, int side, int32_t layer, float *out, st::Attn
   p->norm_k = ctx->d_norm ? ctx->d_norm + (size_t)layer * 256 + 128 : nullptr;
   p->norm_eps = ctx->cfg.qk_norm_eps;
   p->total_work = p->work_per_cta = p->n_cta = 0;
+  p->reverse = 0;
   p->split_o = ctx->split_o[side];
   p->split_ml = ctx->split_ml[side];
   p->split_ticket = ctx->split_ticket[side];
@@ -579,6 +582,7 @@ int launch_attention_entries(st_ctx *ctx, int kind, int32_t layer, const std::ve
       ST_CUDA(ctx, st::launch_attn_reference(ap, total_rows, stream));
       nl = 1;
     } else if (kind == 1) {
+      ap.reverse = ctx->pend[1].reverse ? 1 : 0;
       ST_CUDA(ctx, st::launch_decode(ap, ctx->num_sms, stream, &nl, t0, t1));
     } else {
       ST_CUDA(ctx, st::launch_attn_tc(ap, ctx->precise_p, ctx->num_sms, stream, &nl, t0, t1));
@@ -672,6 +676,8 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     pd.rope_off = off;
     pd.is_final = fin;
     pd.wait_serial = wait_serial;
+    // consecutive decode steps walk the caches in opposite directions: a step starts on what the last one left in L2
+    pd.reverse = kind == 1 && (ctx->decode_steps++ & 1u) != 0;
     record_meta(ctx, kind, seq_ids, cu, n_seq, pd.vis_tokens, pd.rope_off);
   }
 
@@ -1068,6 +1074,7 @@ int st_reset(st_ctx *ctx, const int32_t *seq_ids, int32_t n_seq) {
     for (int i = 0; i < n_seq; ++i) reset_one(seq_ids[i]);
   }
   ctx->pend[0].active = ctx->pend[1].active = false;
+  if (n_seq == 0) ctx->decode_steps = 0;
   if (n_seq == 0) ctx->cross_stream = false;   // a full reset (which waited for the device) starts in single-stream mode again
   if (fill_err != cudaSuccess) return fail(ctx, ST_ERR_CUDA, std::string("sentinel fill: ") + cudaGetErrorString(fill_err));
   if (ctx->poison && !ctx->host_only) ST_CUDA(ctx, cudaDeviceSynchronize());

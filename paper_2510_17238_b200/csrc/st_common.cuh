@@ -108,6 +108,7 @@ struct AttnParams {
   int32_t n_seq, n_q_heads, n_kv_heads, group;
   int32_t total_work;              // total tiles (decode) / blocks (prefill)
   int32_t work_per_cta;            // decode: tiles per CTA
+  int32_t reverse;                 // decode: every CTA walks its slice of the tile list from the end to the start
   int32_t n_cta;
   float scale_log2;                // softmax scale * log2(e)
   double inv_freq[64];             // theta^(-2c/128): the tensor-core kernel rotates its queries itself (from q_raw)
