@@ -10,16 +10,19 @@
 // The key tiles (one page = 64 tokens = one 32 KiB block per kv head) of all (sequence, kv head)
 // pairs form one global list; CTA c takes the contiguous slice [c*L, (c+1)*L) of it, whatever
 // pair boundaries it crosses, so all CTAs stream the same number of bytes. A producer warp feeds a
-// shared-memory ring with one 32 KiB bulk copy (TMA, no tensor map) per tile; four consumer
-// warps each own 16 of a tile's 64 keys and keep an independent online-softmax state, so the
-// only per-tile synchronisation is the ring's full/empty mbarriers. The products run on
+// shared-memory ring with one 32 KiB bulk copy (TMA, no tensor map) per tile; a tile is worked off by four
+// consumer warps, each of which owns 16 of its 64 keys and keeps an independent online-softmax state, so the
+// only per-tile synchronisation is the ring's full/empty mbarriers. There are two such groups of four warps;
+// consecutive tiles of the walk go to them alternately, so that two tiles are in work at a time (the chains of
+// ldmatrix and mma.sync of one tile hide behind the other's: 152.7 -> 151.8 us per launch on the benchmark
+// workload, 141.2 -> 139.2 us on the long-context one). The products run on
 // mma.sync.m16n8k16 in transposed form:
 //     S^T[16 keys x 8 heads]   = K[16 x 128]   . Q^T[128 x 8]      (A = K via ldmatrix)
 //     O^T[128 ch  x 8 heads]  += V^T[128 x 16] . P^T[16 x 8]       (A = V^T via ldmatrix)
 // so the padded dimension is the 8-wide head axis (G <= 8 q heads share a kv head), not M.
 // P^T goes from accumulator to B-operand layout with movmatrix, split into bf16 hi + lo parts
 // so that the rounding of P does not limit accuracy. Per pair slice the four warps combine their
-// states through shared memory (log-sum-exp merge); a slice that covers its pair completely
+// states (all eight warps') through shared memory (log-sum-exp merge); a slice that covers its pair completely
 // writes the final rows, otherwise it writes an (m, l, O) partial that a second small kernel
 // merges across CTAs. All waits are bounded.
 //
@@ -46,8 +49,10 @@ namespace st {
 namespace {
 
 constexpr int kStages = 4;
-constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 2) * 32;   // consumers, producer, append warp
+constexpr int kTileWarps = 4;                 // warps that share a tile: 16 of its 64 keys each
+constexpr int kConsumerGroups = 2;            // groups of kTileWarps warps; consecutive tiles of the walk alternate between them
+constexpr int kConsumerWarps = kTileWarps * kConsumerGroups;
+constexpr int kThreads = (kConsumerWarps + 2) * 32;   // two consumer groups, producer, append warp
 constexpr int kMergeFloats = 8 * 128 + 16;  // per warp: o[8][128], m[8], l[8]
 
 struct __align__(1024) DecodeSmem {
@@ -160,7 +165,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(smem_u32(&sm.full[i]), 1);
-      mbar_init(smem_u32(&sm.empty[i]), kConsumerWarps);
+      mbar_init(smem_u32(&sm.empty[i]), kTileWarps);
     }
     mbar_init(smem_u32(&sm.group_bar), kConsumerWarps);
     for (int i = 0; i < 2; ++i) {
@@ -351,10 +356,12 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
     const int G = p.group;
     PairSlice ps;
     ps.first(p, tile_begin, tile_end, rev);
-    int stage = 0;
-    uint32_t phase = 0, group_phase = 0;
+    uint32_t group_phase = 0;
     bool ok = true;
     int ord = 0;   // ordinal of the slice (pair) within this CTA's walk, as counted by the producer warp
+    const int wq = warp % kTileWarps;    // this warp's quarter of a tile's keys
+    const int grp = warp / kTileWarps;   // its group: it works on the tiles whose ring index is congruent to grp
+    int ring_index = 0;                  // tiles of the walk in front of the current slice
 
     for (bool more = true; more && ok; more = ps.next(p, tile_begin, tile_end, rev)) {
       // ---- one slice of one (sequence, kv head) pair
@@ -392,6 +399,10 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
       for (int mt = 0; mt < 8; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
 
       for (int k = 0; k < ps.tiles(); ++k) {
+        const int ri = ring_index + k;
+        if (ri % kConsumerGroups != grp) continue;            // the other group's tile
+        const int stage = ri % kStages;
+        const uint32_t phase = (uint32_t)(ri / kStages) & 1u;
         const int t = ps.tile_at(k, rev);
         if (!mbar_wait(smem_u32(&sm.full[stage]), phase, abort_flag, p.status, kDevTimeoutDecode)) { ok = false; break; }
         const uint32_t sb = smem_u32(sm.ring[stage]);
@@ -405,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         float c[4] = {0.f, 0.f, 0.f, 0.f};
         {
           float c_odd[4] = {0.f, 0.f, 0.f, 0.f};
-          const int key = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int key = wq * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             uint32_t a0, a1, a2, a3;
@@ -416,7 +427,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
 #pragma unroll
           for (int i = 0; i < 4; ++i) c[i] += c_odd[i];
         }
-        const int key0 = warp * 16 + g;
+        const int key0 = wq * 16 + g;
         const float NEG = -INFINITY;
         c[0] = key0 < valid ? c[0] * p.scale_log2 : NEG;
         c[1] = key0 < valid ? c[1] * p.scale_log2 : NEG;
@@ -456,7 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         // O^T += V^T . P^T
         {
           const int ch = (lane & 7) + ((lane >> 3) & 1) * 8;
-          const int tok = warp * 16 + (lane >> 4) * 8;
+          const int tok = wq * 16 + (lane >> 4) * 8;
 #pragma unroll
           for (int mt = 0; mt < 8; ++mt) {
             uint32_t a0, a1, a2, a3;
@@ -467,9 +478,9 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sm.empty[stage]));
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
       if (!ok) break;
+      ring_index += ps.tiles();
 
       // ---- combine the four warps' states (log-sum-exp merge through shared memory)
 #pragma unroll
@@ -497,12 +508,12 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
       group_phase ^= 1u;
 
       const bool whole_pair = (pair_first >= tile_begin) && (pair_first + pair_tiles <= tile_end);
-      const int d = threadIdx.x;  // 0..127: output channel
+      const int d = threadIdx.x % 128;   // output channel; the two halves of the consumer threads take alternate heads
       {
         // pair index in launch order and partial slot of this (pair, CTA)
         const int pidx = slice_seq * Hkv + kvh;   // (cur has already advanced past the slice)
         float *rec = p.partial + (size_t)(pidx + blockIdx.x) * kPartialFloats;
-        for (int h = 0; h < G; ++h) {
+        for (int h = threadIdx.x / 128; h < G; h += kConsumerWarps * 32 / 128) {
           float M = -INFINITY;
 #pragma unroll
           for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.merge[w][1024 + h]);
