@@ -66,7 +66,8 @@ def test_ragged_edges(hq):
         assert pu.check_cache(ctx, w, scheds, plan, flats[0]) <= 2
 
 
-@pytest.mark.parametrize("hq,variant", [(8, "plain"), (32, "plain"), (40, "plain"), (40, "two_term"), (16, "qk_norm")])
+@pytest.mark.parametrize("hq,variant", [(8, "plain"), (32, "plain"), (40, "plain"), (40, "two_term"), (16, "qk_norm"),
+                                        (32, "two_streams")])
 def test_key_split_of_long_items(hq, variant):
     """Work items of twenty and more cache pages in a launch that fills less than half of the SMs: the tensor-core
     kernel cuts each of them in two by keys and the part that finishes second merges. Twenty pages exactly and
@@ -84,7 +85,9 @@ def test_key_split_of_long_items(hq, variant):
     if variant == "qk_norm":
         rng = np.random.default_rng(5)
         norm = (rng.uniform(0.5, 1.5, size=(1, 128)).astype(np.float32), rng.uniform(0.5, 1.5, size=(1, 128)).astype(np.float32), 1e-6)
-    ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode="extend", lookahead=1, cfg_flags=flags, qk_norm=norm)
+    # (two_streams: the chunk prefills on one stream, the spans on another; each side has its own merge workspace)
+    ctx, plan, batches, flats = pu.run_plan(w, scheds, 0, mode="extend", lookahead=1, cfg_flags=flags, qk_norm=norm,
+                                            two_streams=variant == "two_streams")
     norm0 = None if norm is None else (norm[0][0], norm[1][0], norm[2])
     worst = pu.check_against_oracle(w, scheds, plan, batches[0], flats[0], n_random=160, what=f"key split hq={hq} {variant}",
                                     qk_norm=norm0)
