@@ -350,7 +350,9 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
   // Q rows of M-tile t into the swizzled operand layout, by asynchronous 16-byte copies: the tile's 128 threads copy it
   // 8 rows at a time, 16 lanes take the 16 chunks of one row, so every copy instruction reads whole 256-byte rows; rows
   // past the end of the sequence are zero-filled (source size 0, nothing is read).
-  auto issue_q_copies = [&](int t, int r_local) {
+  // `between(i)` runs behind copy i: the copy instructions stall at issue once enough of them are in flight, so work that
+  // needs no memory is placed between them instead of behind them.
+  auto issue_q_copies = [&](int t, int r_local, auto between) {
     const __nv_bfloat16 *q_src = kPrecise ? p.qhat : p.q_raw;
     const int c = r_local & 15;                            // chunk of the row
     const uint32_t q_smem = smem_u32(smem + kOffQ + t * kQTileBytes);
@@ -362,12 +364,28 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       const bool in = grow < packed_rows;
       const __nv_bfloat16 *src = in ? q_src + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + c * 8 : q_src;
       cp_async16(q_smem + (c >> 3) * kHalfPanel + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src, in ? 16u : 0u);
+      between(i);
     }
   };
   // The one-term variant reads the caller's un-rotated queries, which no kernel in front of this one writes: their
-  // copies start at once and fly while the barriers and the tensor memory are set up (about 2,000 cycles).
+  // copies start at once and fly while the barriers and the tensor memory are set up. Between the copies each thread
+  // computes the rotation angles of its first two work items of the rotation pass below (item = (token, chunk c): 8
+  // angles; all items up to 32 tokens per M-tile, i.e. from 4 query heads per kv head on): the copy instructions of
+  // a thread take ~3,000 cycles to issue (per-CTA trace), and the angles ride along for a few hundred more.
+  float cs_pre[2][8], sn_pre[2][8];
   if constexpr (!kPrecise) {
-    if (warp < 8 && active[warp >> 2]) issue_q_copies(warp >> 2, (warp & 3) * 32 + lane);
+    if (warp < 8 && active[warp >> 2]) {
+      const int t = warp >> 2, r_local = (warp & 3) * 32 + lane;
+      const int tok_first = div_g(row0 + t * kRowsPerTile);
+      issue_q_copies(t, r_local, [&](int i) {
+        const int it = r_local + (i >> 3) * kRowsPerTile, e = i & 7;   // angle e of item `it` (see the rotation pass)
+        const double pos = (double)(sq.b_base + tok_first + (it >> 3) + sq.rope_off);
+        const double turns = pos * p.inv_freq[8 * (it & 7) + e] * 0.15915494309189535;   // angle / 2 pi
+        const float r = (float)(turns - rint(turns)) * 6.2831853071795865f;              // in [-pi, pi]
+        sn_pre[i >> 3][e] = sin_approx(r);
+        cs_pre[i >> 3][e] = cos_approx(r);
+      });
+    }
   }
 
   // one thread per barrier (24 of them: a single thread took ~600 cycles over this). Barriers that the four softmax
@@ -432,15 +450,9 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           cs[e] = cos_approx(r);
         }
       };
-      // The angles of this thread's first two items (all of them up to 32 tokens per M-tile, i.e. from 4 query heads
-      // per kv head on) need no memory: they are computed while the query copies are in flight.
-      float cs_pre[2][8], sn_pre[2][8];
-      if constexpr (!kPrecise) {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) item_angles(r_local + i * kRowsPerTile, cs_pre[i], sn_pre[i]);
-      }
+      // (the angles of this thread's first two items were computed between the query copies, before the set-up)
       {
-        if constexpr (kPrecise) issue_q_copies(t, r_local);   // (the one-term variant issued them before the set-up)
+        if constexpr (kPrecise) issue_q_copies(t, r_local, [](int) {});   // (the one-term variant issued them before the set-up)
         cp_async_wait_all();
       }
       if constexpr (!kPrecise) {
