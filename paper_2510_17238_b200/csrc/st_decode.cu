@@ -53,7 +53,12 @@ constexpr int kTileWarps = 4;                 // warps that share a tile: 16 of 
 constexpr int kConsumerGroups = 2;            // groups of kTileWarps warps; consecutive tiles of the walk alternate between them
 constexpr int kConsumerWarps = kTileWarps * kConsumerGroups;
 constexpr int kThreads = (kConsumerWarps + 2) * 32;   // two consumer groups, producer, append warp
-constexpr int kMergeFloats = 8 * 128 + 16;  // per warp: o[8][128], m[8], l[8]
+// Per warp: o[8][128] with the head rows kMergeRow floats apart (132: the four lanes of a quad write heads 2 tq, i.e.
+// rows 264 tq floats = 8 tq banks apart, and the stores are conflict-free; with rows of 128 they were 4-way conflicts),
+// then m[8], l[8].
+constexpr int kMergeRow = 132;
+constexpr int kMergeM = 8 * kMergeRow, kMergeL = kMergeM + 8;
+constexpr int kMergeFloats = kMergeL + 8;
 
 struct __align__(1024) DecodeSmem {
   uint8_t ring[kStages][kBlockBytes];
@@ -491,16 +496,16 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
       float *mg = sm.merge[warp];
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
-        mg[(2 * tq) * 128 + mt * 16 + g] = o[mt][0];
-        mg[(2 * tq + 1) * 128 + mt * 16 + g] = o[mt][1];
-        mg[(2 * tq) * 128 + mt * 16 + g + 8] = o[mt][2];
-        mg[(2 * tq + 1) * 128 + mt * 16 + g + 8] = o[mt][3];
+        mg[(2 * tq) * kMergeRow + mt * 16 + g] = o[mt][0];
+        mg[(2 * tq + 1) * kMergeRow + mt * 16 + g] = o[mt][1];
+        mg[(2 * tq) * kMergeRow + mt * 16 + g + 8] = o[mt][2];
+        mg[(2 * tq + 1) * kMergeRow + mt * 16 + g + 8] = o[mt][3];
       }
       if (g == 0) {
-        mg[1024 + 2 * tq] = m0;
-        mg[1024 + 2 * tq + 1] = m1;
-        mg[1032 + 2 * tq] = l0;
-        mg[1032 + 2 * tq + 1] = l1;
+        mg[kMergeM + 2 * tq] = m0;
+        mg[kMergeM + 2 * tq + 1] = m1;
+        mg[kMergeL + 2 * tq] = l0;
+        mg[kMergeL + 2 * tq + 1] = l1;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&sm.group_bar));
@@ -516,13 +521,13 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_decode(const __grid_constant
         for (int h = threadIdx.x / 128; h < G; h += kConsumerWarps * 32 / 128) {
           float M = -INFINITY;
 #pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.merge[w][1024 + h]);
+          for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.merge[w][kMergeM + h]);
           float L = 0.f, O = 0.f;
 #pragma unroll
           for (int w = 0; w < kConsumerWarps; ++w) {
-            const float f = exp2f(sm.merge[w][1024 + h] - M);   // a warp that saw no valid key has m = -inf -> 0
-            L += sm.merge[w][1032 + h] * f;
-            O += sm.merge[w][h * 128 + d] * f;
+            const float f = exp2f(sm.merge[w][kMergeM + h] - M);   // a warp that saw no valid key has m = -inf -> 0
+            L += sm.merge[w][kMergeL + h] * f;
+            O += sm.merge[w][h * kMergeRow + d] * f;
           }
           if (whole_pair) {
             p.out[((size_t)sq.q_begin * p.n_q_heads + (size_t)kvh * G + h) * kHeadDim + d] = O / L;
