@@ -138,7 +138,11 @@ typedef struct st_config {
 ST_API uint64_t st_pool_bytes(const st_config *cfg);
 
 /* Create a context (Algorithm 1, line 1: initialise the caches). Allocates page tables, scratch
- * and, if cfg->pool_base is NULL, the pools; zero-fills the pools. `*out` is set on success. */
+ * and, if cfg->pool_base is NULL, the pools; zero-fills the pools. `*out` is set on success.
+ * Scratch besides the pools: the split-K records of the decode kernel (a few MB), two rotation tables, per side a
+ * rotated-query buffer of max_tokens_per_call rows and 19.5 MB in which the attention kernel's key-split halves meet
+ * (two CTAs share a long work item when the last wave of a launch would leave SMs idle); host-I/O staging buffers
+ * are allocated by the first call that needs them. */
 ST_API int st_create(const st_config *cfg, st_ctx **out);
 
 /* Wait for the device, then free everything the context owns (never cfg->pool_base). */
