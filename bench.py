@@ -36,10 +36,10 @@ import numpy as np
 import torch
 
 # DRAM bytes per algorithmic byte of st_k_decode, from an ncu capture of the small decode case (--profile-case decode:
-# 273.5 MB moved on average for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to
+# 274.0 MB moved on average for 268.6 MB of K/V, query and output): a full-size launch holds too much memory to
 # capture. The profiler flushes the caches in front of every launch; in the real run a step finds up to ~50 MB of the
 # step before it in L2 (the steps walk the caches in alternating directions), so the real traffic is a little lower.
-DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.018
+DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.020
 # The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 191.2 and 202.2 MB moved for 209.7
 # and 220.2 MB of K/V, queries and output rows; below 1 because the rows a launch writes are still in L2 when it ends).
 PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.915
