@@ -764,9 +764,8 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
   } else if (warp == kProducerWarp) {
     // =========================================================== producer
     if (lane == 0) {
-      for (int j = 0; j < n_max; ++j) {
-        const int n_pg = min(2, n_pages - 2 * j);              // pages of this tile: 2, or 1 in an odd tail
-        const uint8_t *src[2];
+      // blocks of the (one or two) pages of key tile j; false if a page id lies outside its pool
+      auto tile_pages = [&](int j, const uint8_t *(&src)[2]) -> bool {
         bool pages_ok = true;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -777,28 +776,60 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
           pages_ok = pages_ok && page_ok(page, in_a ? p.n_pages_a : p.n_pages_b, abort_flag, p.status);
           src[h] = (in_a ? p.pool_a : p.pool_b) + ((size_t)page * Hkv + kvh) * kBlockBytes;
         }
-        if (!pages_ok) break;   // nothing is copied from an address built on a bad page id
-        {
-          const int st = j % kKStages;
-          const uint32_t use = (uint32_t)(j / kKStages);
-          if (!mbar_wait(smem_u32(&bar.k_empty[st]), (use & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutPrefill)) break;
-          const uint32_t full = smem_u32(&bar.k_full[st]);
-          const uint32_t dst = smem_u32(smem + kOffK + st * kKStageBytes);
-          mbar_arrive_expect_tx(full, (uint32_t)(n_pg * kKeyBytes));
-          for (int h = 0; h < n_pg; ++h) {
-            // channel half c of page h -> rows 64h .. 64h+63 of the stage's panel c
-            bulk_load(dst + h * kPanelBytesK, src[h], kPanelBytesK, full);
-            bulk_load(dst + kHalfPanel + h * kPanelBytesK, src[h] + kPanelBytesK, kPanelBytesK, full);
-          }
+        return pages_ok;   // nothing is copied from an address built on a bad page id
+      };
+      auto pages_of = [&](int j) { return min(2, n_pages - 2 * j); };   // 2, or 1 in an odd tail
+      auto wait_k_stage = [&](int j) {
+        const uint32_t use = (uint32_t)(j / kKStages);
+        return mbar_wait(smem_u32(&bar.k_empty[j % kKStages]), (use & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutPrefill);
+      };
+      auto wait_v_stage = [&](int j) {
+        const uint32_t use = (uint32_t)(j / kVStages);
+        return mbar_wait(smem_u32(&bar.v_empty[j % kVStages]), (use & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutPrefill);
+      };
+      auto copy_k = [&](int j, const uint8_t *const (&src)[2], uint32_t full) {
+        const uint32_t dst = smem_u32(smem + kOffK + (j % kKStages) * kKStageBytes);
+        for (int h = 0; h < pages_of(j); ++h) {
+          // channel half c of page h -> rows 64h .. 64h+63 of the stage's panel c
+          bulk_load(dst + h * kPanelBytesK, src[h], kPanelBytesK, full);
+          bulk_load(dst + kHalfPanel + h * kPanelBytesK, src[h] + kPanelBytesK, kPanelBytesK, full);
         }
-        {
-          const int st = j % kVStages;
-          const uint32_t use = (uint32_t)(j / kVStages);
-          if (!mbar_wait(smem_u32(&bar.v_empty[st]), (use & 1u) ^ 1u, abort_flag, p.status, kDevTimeoutPrefill)) break;
-          const uint32_t full = smem_u32(&bar.v_full[st]);
-          const uint32_t dst = smem_u32(smem + kOffV + st * kVStageBytes);
-          mbar_arrive_expect_tx(full, (uint32_t)(n_pg * kHalfPanel));
-          for (int h = 0; h < n_pg; ++h) bulk_load(dst + h * kHalfPanel, src[h] + kKeyBytes, kHalfPanel, full);
+      };
+      auto copy_v = [&](int j, const uint8_t *const (&src)[2], uint32_t full) {
+        const uint32_t dst = smem_u32(smem + kOffV + (j % kVStages) * kVStageBytes);
+        for (int h = 0; h < pages_of(j); ++h) bulk_load(dst + h * kHalfPanel, src[h] + kKeyBytes, kHalfPanel, full);
+      };
+      if constexpr (kPrecise) {
+        // one K stage: K(j) and V(j) of a tile, each on its own barrier
+        for (int j = 0; j < n_max; ++j) {
+          const uint8_t *src[2];
+          if (!tile_pages(j, src)) break;
+          if (!wait_k_stage(j)) break;
+          mbar_arrive_expect_tx(smem_u32(&bar.k_full[j % kKStages]), (uint32_t)(pages_of(j) * kKeyBytes));
+          copy_k(j, src, smem_u32(&bar.k_full[j % kKStages]));
+          if (!wait_v_stage(j)) break;
+          mbar_arrive_expect_tx(smem_u32(&bar.v_full[j % kVStages]), (uint32_t)(pages_of(j) * kHalfPanel));
+          copy_v(j, src, smem_u32(&bar.v_full[j % kVStages]));
+        }
+      } else {
+        // K(0) on its own barrier; then V(j) and K(j+1) together on v_full[j % 2]: the issuer needs both at the same
+        // point of tile j (P V (j, 0), then Q K^T (j+1)), and every wait it does not have to make is ~400 cycles.
+        const uint8_t *cur[2], *nxt[2];
+        bool ok = n_max > 0 && tile_pages(0, cur) && wait_k_stage(0);
+        if (ok) {
+          mbar_arrive_expect_tx(smem_u32(&bar.k_full[0]), (uint32_t)(pages_of(0) * kKeyBytes));
+          copy_k(0, cur, smem_u32(&bar.k_full[0]));
+        }
+        for (int j = 0; ok && j < n_max; ++j) {
+          const bool more = j + 1 < n_max;
+          if (more && !tile_pages(j + 1, nxt)) break;
+          if (!wait_v_stage(j) || (more && !wait_k_stage(j + 1))) break;
+          const uint32_t full = smem_u32(&bar.v_full[j % kVStages]);
+          mbar_arrive_expect_tx(full, (uint32_t)(pages_of(j) * kHalfPanel + (more ? pages_of(j + 1) * kKeyBytes : 0)));
+          copy_v(j, cur, full);
+          if (more) copy_k(j + 1, nxt, full);
+          cur[0] = nxt[0];
+          cur[1] = nxt[1];
         }
       }
     }
@@ -874,7 +905,13 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
       bool have_k = false;
       for (int t = 0; t < 2 && ok; ++t) {
         if (j >= n_tiles[t]) continue;
-        ok = mbar_wait(smem_u32(&bar.p_full[t][0]), (uint32_t)j & 1u, abort_flag, p.status, kDevTimeoutPrefill);
+        // With two key halves one wait serves P V (j, 0) and Q K^T (j+1): every softmax warp arrives at y_loaded
+        // behind its arrival at p_full[0] (program order, both releases), so a complete y_loaded phase means that P of
+        // half 0 is published as well. Every wait of this warp costs ~400 cycles while MMAs run (its polls are
+        // shared-memory accesses in competition with the operand reads), and the issuer's chain of waits was the
+        // longest path through a key tile (per-CTA trace: nine steps of 370-400 cycles).
+        ok = halves == 2 ? mbar_wait(smem_u32(&bar.y_loaded[t]), (uint32_t)j & 1u, abort_flag, p.status, kDevTimeoutPrefill)
+                         : mbar_wait(smem_u32(&bar.p_full[t][0]), (uint32_t)j & 1u, abort_flag, p.status, kDevTimeoutPrefill);
         if (ok && t == (n_tiles[0] > j ? 0 : 1))
           ok = mbar_wait(smem_u32(&bar.v_full[j % kVStages]), (uint32_t)(j / kVStages) & 1u, abort_flag, p.status, kDevTimeoutPrefill);
         if (!ok) break;
@@ -883,10 +920,8 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         tc_commit(smem_u32(&bar.pv0_done[t]), issue);
         if (halves == 1 && j == n_tiles[t] - 1) tc_commit(smem_u32(&bar.o_final[t]), issue);
         if (halves == 2) {
-          ok = mbar_wait(smem_u32(&bar.y_loaded[t]), (uint32_t)j & 1u, abort_flag, p.status, kDevTimeoutPrefill);
-          if (!ok) break;
           if (j + 1 < n_tiles[t]) {
-            if (!have_k) {
+            if (kPrecise && !have_k) {   // (one-term variant: K(j+1) came with V(j), on the barrier waited for above)
               ok = mbar_wait(smem_u32(&bar.k_full[(j + 1) % kKStages]), (uint32_t)((j + 1) / kKStages) & 1u, abort_flag, p.status, kDevTimeoutPrefill);
               have_k = true;
               if (!ok) break;
