@@ -78,7 +78,7 @@ extern "C" {
 #define ST_REFERENCE_KERNELS   2u  /* run the slow, simple attention kernels instead of the tuned ones    */
 #define ST_IO_HOST             4u  /* q/k/v/out are HOST pointers (page-locked memory recommended). A large
                                       call copies them to and from internal device staging on `stream`; a
-                                      call whose q + k + v stay below 1 MiB (a decode step) and whose buffers
+                                      st_reason_decode call whose q + k + v stay below 1 MiB and whose buffers
                                       are all page-locked is served in place: its kernels read q/k/v and
                                       write the rows directly in host memory. Either way the buffers belong
                                       to the call until the work queued on `stream` has completed            */

@@ -405,8 +405,10 @@ const void *device_alias_of_host(const void *p) {
 // transfers of that size cost more than the attention itself, so when all buffers are page-locked the append
 // kernel reads q/k/v, and the attention kernels write the rows, directly in host memory -- each byte crosses the
 // bus once, inside the kernels of the call.
+// `may_run_in_place`: small calls on page-locked buffers may be served by the kernels themselves (decode steps only:
+// the tensor-core attention kernel writes its rows with bulk stores from shared memory, which are kept to device memory).
 int stage_inputs(st_ctx *ctx, int side, uint32_t flags, int32_t total, const void *q, const void *k, const void *v,
-                 void *out, cudaStream_t stream, IoPtrs *io) {
+                 void *out, cudaStream_t stream, IoPtrs *io, bool may_run_in_place) {
   io->q = (const __nv_bfloat16 *)q;
   io->k = (const __nv_bfloat16 *)k;
   io->v = (const __nv_bfloat16 *)v;
@@ -414,7 +416,7 @@ int stage_inputs(st_ctx *ctx, int side, uint32_t flags, int32_t total, const voi
   if (int rc = injected_failure(ctx, "staging copy")) return rc;
   if (!(flags & ST_IO_HOST) || ctx->host_only || total == 0) return ST_OK;
   const size_t qb = (size_t)total * ctx->cfg.n_q_heads * 256, kb = (size_t)total * ctx->cfg.n_kv_heads * 256;
-  if (qb + 2 * kb <= kInPlaceHostIoBytes) {
+  if (may_run_in_place && qb + 2 * kb <= kInPlaceHostIoBytes) {
     const void *dq = device_alias_of_host(q), *dk = device_alias_of_host(k), *dv = device_alias_of_host(v);
     const void *dout = out ? device_alias_of_host(out) : nullptr;
     if (dq && dk && dv && (dout || !out)) {
@@ -690,7 +692,7 @@ int attention_call(st_ctx *ctx, int kind, int32_t layer, const int32_t *seq_ids,
     if (kind != 0 && (r = wait_for_append(ctx, pd.wait_serial, stream))) return r;
     if ((r = push_page_updates(ctx, updates, stream))) return r;
     IoPtrs io;
-    if ((r = stage_inputs(ctx, side, flags, total, q, k, v, out, stream, &io))) return r;
+    if ((r = stage_inputs(ctx, side, flags, total, q, k, v, out, stream, &io, kind == 1))) return r;
     // A decode step's append (one token per sequence) runs inside the decode kernel: the step is then two kernels
     // instead of three. Cache-only calls and the cross-check kernels keep the separate append.
     const bool fuse_append = kind == 1 && io.out != nullptr && !(flags & ST_REFERENCE_KERNELS) && !ctx->host_only;
@@ -847,7 +849,7 @@ int forward_packed(st_ctx *ctx, int32_t layer, const int32_t *seq_ids, int32_t n
     if (!ctx->host_only) ST_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     if ((r = push_page_updates(ctx, updates, stream))) return r;
     IoPtrs io;
-    if ((r = stage_inputs(ctx, 0, flags, (int32_t)total, q, k, v, out, stream, &io))) return r;
+    if ((r = stage_inputs(ctx, 0, flags, (int32_t)total, q, k, v, out, stream, &io, false))) return r;
     const bool want_qhat = io.out != nullptr && ((flags & ST_REFERENCE_KERNELS) || ctx->precise_p);
     RowRanges src_rows, rsn_rows;
     for (int b = 0; b < n_seq; ++b) {

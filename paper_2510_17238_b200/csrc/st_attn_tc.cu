@@ -83,6 +83,9 @@ constexpr int kOffV = kOffK + kKStagesFast * kKStageBytes;
 constexpr int kOffP1 = kOffV + kVStages * kVStageBytes;   // P of the second key half, per M-tile: 128 rows x 64 keys bf16
 constexpr int kP1Bytes = 16384;
 constexpr int kOffBar = kOffP1 + 2 * kP1Bytes;
+// epilogue staging (over the Q buffers and the start of the first K stage): one line per row
+constexpr int kOutStageLine = 272, kOutStageTile = 36864;
+static_assert(kOutStageTile >= kRowsPerTile * kOutStageLine && kOutStageTile + kRowsPerTile * kOutStageLine <= kOffK + kKStageBytes, "epilogue staging");
 constexpr int kSmemBytes = kOffBar + 256;
 static_assert(kSmemBytes + 1024 <= 232448, "shared memory budget of one CTA");
 
@@ -159,6 +162,13 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
       : "memory");
 }
+// One bulk store shared -> global (TMA, no tensor map): both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// until the bulk stores of this thread have read their shared-memory source
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -666,16 +676,22 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
         }
       }
 
-      // ---- epilogue: O / l to global memory, through the tile's own Q buffer (no MMA reads it any more once the
-      // last P V is complete) so that every store instruction writes whole rows. Two passes of 64 channels:
-      // thread = row writes its 256 bytes as 16 chunks, chunk c at position c ^ (row & 15) (conflict-free); then
-      // 16 lanes take one row each time and write it out contiguously. All four warps of the tile run both
-      // passes whatever happened before, so the group barrier cannot be left waiting.
+      // ---- epilogue: O / l to global memory (write_rows below). All four warps of the tile take the same path whatever
+      // happened before.
       const bool fin = ok && mbar_wait(smem_u32(&bar.o_final[t]), 0, abort_flag, p.status, kDevTimeoutPrefill);
       tc_fence_after();
-      uint8_t *stage = smem + kOffQ + t * kQTileBytes;        // 128 rows x 256 bytes
       // The tile's accumulator to the output rows: this thread's row times `mul`; with `other` set, plus the other
-      // part's share of the row (workspace, in the layout of write_share below) times `other_mul`.
+      // part's share of the row (workspace, in the layout of write_share below) times `other_mul`. Thread = row: the
+      // thread lays 64 channels of its row (256 bytes) into its own line of a staging area and hands the line to the
+      // TMA unit as one bulk store, so the rows leave in 256-byte pieces without a transpose between threads, without
+      // group barriers and without store instructions of the warps. Lines are 272 bytes apart (the 32 lanes of a
+      // 16-byte store then hit every bank group four times, the minimum). The staging area lies over shared memory
+      // that no MMA reads any more once the tile's last P V is complete: M-tile 0 its own Q buffer and the first 2 KiB
+      // of M-tile 1's (whose last score product was issued in front of this tile's last P V), M-tile 1 the rest of
+      // its Q buffer and the start of the first K stage.
+      uint8_t *my_line = smem + kOffQ + t * kOutStageTile + r_local * kOutStageLine;
+      float *out_row = p.out + ((size_t)(sq.q_begin + tok) * Hq + (size_t)(kvh * G + (row - tok * G))) * kHeadDim;
+      const bool store_row = fin && row < packed_rows;
       auto write_rows = [&](float mul, const float4 *other, float other_mul) {
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -689,6 +705,7 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
               for (int c = 0; c < 8; ++c) o[c] = __ldcg(other + (size_t)((half * 64 + c0) / 4 + c) * kRowsPerTile + r_local);
             }
             tmem_wait_ld();
+            if (half == 1 && c0 == 0) bulk_store_wait_read();   // the line is free again once the first half has been read
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
               // (each product is rounded on its own - no fused multiply-add - and the sum commutes: the bits do not
@@ -699,23 +716,14 @@ __global__ void __launch_bounds__(kThreads, 1) st_k_attn_tc(const __grid_constan
                 v = make_float4(__fadd_rn(v.x, __fmul_rn(w.x, other_mul)), __fadd_rn(v.y, __fmul_rn(w.y, other_mul)),
                                 __fadd_rn(v.z, __fmul_rn(w.z, other_mul)), __fadd_rn(v.w, __fmul_rn(w.w, other_mul)));
               }
-              *reinterpret_cast<float4 *>(stage + r_local * 256 + ((((c0 + c) >> 2) ^ (r_local & 15)) << 4)) = v;
+              *reinterpret_cast<float4 *>(my_line + (c0 + c) * 4) = v;
             }
           }
-          tile_sync(t);
-          const int c = r_local & 15;
-#pragma unroll 4
-          for (int i = 0; i < 16; ++i) {
-            const int rr = i * 8 + (r_local >> 4);
-            const int grow = row0 + t * kRowsPerTile + rr;
-            const float4 v = *reinterpret_cast<const float4 *>(stage + rr * 256 + ((c ^ (rr & 15)) << 4));
-            if (fin && grow < packed_rows) {
-              const int gt = div_g(grow), gh = kvh * G + (grow - gt * G);
-              *reinterpret_cast<float4 *>(p.out + ((size_t)(sq.q_begin + gt) * Hq + gh) * kHeadDim + half * 64 + c * 4) = v;
-            }
-          }
-          tile_sync(t);
+          fence_proxy_async_smem();
+          if (store_row) bulk_store(out_row + half * 64, smem_u32(my_line), 256);
+          bulk_store_commit();
         }
+        bulk_store_wait_read();
       };
       // This part's un-normalised share of the tile to the workspace, straight from tensor memory: 16-byte chunk q of
       // row r at [q][r], so that a warp's 32 rows write (and the merging part reads) 512 contiguous bytes.
