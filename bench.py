@@ -40,9 +40,9 @@ import torch
 # capture. The profiler flushes the caches in front of every launch; in the real run a step finds up to ~50 MB of the
 # step before it in L2 (the steps walk the caches in alternating directions), so the real traffic is a little lower.
 DECODE_DRAM_PER_ALGORITHMIC_BYTE = 1.020
-# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 191.7 and 203.3 MB moved for 209.7
+# The same ratio for st_k_attn_tc from the small prefill case (--profile-case prefill: 191.6 and 202.4 MB moved for 209.7
 # and 220.2 MB of K/V, queries and output rows; below 1 because the rows a launch writes are still in L2 when it ends).
-PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.919
+PREFILL_DRAM_PER_ALGORITHMIC_BYTE = 0.916
 
 METRIC = "reasoning-decode tok/s per layer (chunk prefill concurrent on a second stream)"
 UNIT = "tok/s"
